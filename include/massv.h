@@ -1,0 +1,188 @@
+/*
+ * massv.h - C ABI of the target-side verification step of speculative decoding
+ * for vision-language models (MASSV paper, Sec. 2.1) on NVIDIA B200 (sm_100a).
+ *
+ * One verify step, per sequence b of a batch, takes the gamma tokens proposed
+ * by a draft model plus the last emitted token (R = gamma + 1 "block rows"),
+ * scores all of them with the target model in one pass, and decides how many
+ * drafts survive:
+ *
+ *   massv_verify_attn   attention of the R block rows over a paged bf16 KV
+ *                       cache (image-token prefix, then text, then the block),
+ *                       appending the block's K/V to the cache;
+ *   massv_accept        LM-head logits for the R rows, temperature softmax,
+ *                       sequential acceptance of the drafts, the extra token
+ *                       (residual draw on rejection, bonus draw otherwise),
+ *                       accepted length;
+ *   massv_kv_commit     advance (or, on rollback, keep) the cache lengths.
+ *
+ * General rules
+ *   - Every pointer argument except descriptors is DEVICE memory owned by the
+ *     caller and valid until the stream has run the call.  Descriptors are
+ *     host structs read during the call.
+ *   - Calls enqueue work on `stream` and return without synchronising it.  The
+ *     library allocates no device memory; scratch comes from `workspace`
+ *     (256-byte aligned, at least *_workspace_size() bytes, contents undefined
+ *     on entry and exit; two calls that may overlap on the GPU need separate
+ *     workspaces).
+ *   - bf16 tensors are dense, row-major in the index order given, last index
+ *     fastest.  Pointers must be 16-byte aligned.
+ *   - The return value reports errors detectable on the host before anything is
+ *     launched (nothing is enqueued then).  `dev_status`, when not NULL, is one
+ *     int32 the caller zeroes; kernels store a negative massv_status there when
+ *     they detect a problem on the device (an unmapped page, a wait that ran
+ *     out).  It never traps or hangs the GPU.
+ *   - The library draws no random numbers: uniforms are inputs.
+ */
+#ifndef MASSV_H
+#define MASSV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st *massv_stream_t;   /* a cudaStream_t */
+
+typedef enum massv_status {
+    MASSV_OK = 0,
+    MASSV_ERR_INVALID_ARG = -1,   /* NULL where data is required, non-positive size, misaligned pointer */
+    MASSV_ERR_UNSUPPORTED = -2,   /* shape outside the supported set (see each call) */
+    MASSV_ERR_CAPACITY = -3,      /* page table cannot hold L_b + gamma + 1 positions */
+    MASSV_ERR_WORKSPACE = -4,     /* workspace NULL, misaligned or too small */
+    MASSV_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed */
+    MASSV_ERR_TIMEOUT = -6        /* device-side wait exceeded its iteration limit (dev_status only) */
+} massv_status;
+
+/* Geometry of the attention call. */
+typedef struct massv_attn_desc {
+    int32_t batch;               /* B >= 1 */
+    int32_t gamma;               /* speculation length, 0..7; R = gamma + 1 query rows per sequence */
+    int32_t n_q_heads;           /* Hq, a multiple of n_kv_heads; (Hq/Hkv) * R <= 64 */
+    int32_t n_kv_heads;          /* Hkv */
+    int32_t head_dim;            /* d: 64, 128 or 256 */
+    int32_t page_size;           /* tokens per KV page: 16 */
+    int32_t max_pages_per_seq;   /* row length of page_table */
+    int64_t num_pages;           /* pages in the pool */
+    float scale;                 /* score scale; 0 selects 1/sqrt(d) */
+    int32_t kv_chunk;            /* tokens per split of the KV scan, multiple of 64; 0 = choose automatically */
+    uint32_t flags;              /* reserved, 0 */
+} massv_attn_desc;
+
+/* Geometry of the acceptance call. */
+typedef struct massv_accept_desc {
+    int32_t batch;               /* B >= 1; M = B * (gamma + 1) <= 512 rows */
+    int32_t gamma;               /* 0..7 */
+    int32_t hidden;              /* K, a multiple of 64 */
+    int32_t vocab;               /* V, a multiple of 8 */
+    float temperature;           /* T >= 0; 0 selects greedy verification */
+    uint32_t flags;              /* reserved, 0 */
+} massv_accept_desc;
+
+/* Bytes of scratch massv_verify_attn needs for this geometry (0 on a bad descriptor). */
+size_t massv_verify_attn_workspace_size(const massv_attn_desc *desc);
+
+/*
+ * Target attention for the block rows (Sec. 2.1: the target scores positions
+ * t+1 .. t+gamma+1 "in parallel with one forward call"; Sec. 2.2: the context
+ * is m projected image features followed by text tokens).
+ *
+ * For sequence b with committed length L_b = seq_lens[b]:
+ *   1. k_new[b,j], v_new[b,j] are stored at cache position L_b + j (j = 0..gamma)
+ *      through page_table (position i lives in page page_table[b, i / 16],
+ *      slot i % 16).  seq_lens is NOT modified (see massv_kv_commit).
+ *   2. out[b,j,h,:] = sum_i softmax_i(scale * <q[b,j,h,:], K_i>) V_i over
+ *      positions i = 0 .. L_b + j of KV head h / (Hq/Hkv): the whole committed
+ *      prefix and the block rows up to and including j (causal inside the block).
+ * Q and cached K are used as given (any positional encoding is already applied).
+ *
+ *   q                bf16 [B, R, Hq, d]
+ *   k_new, v_new     bf16 [B, R, Hkv, d]
+ *   k_pages, v_pages bf16 [num_pages, Hkv, 16, d]   (written at the block slots)
+ *   page_table       int32 [B, max_pages_per_seq]; entries covering positions
+ *                    0 .. L_b + gamma must be valid page ids
+ *   seq_lens         int32 [B], 0 <= L_b and L_b + R <= 16 * max_pages_per_seq
+ *   out              bf16 [B, R, Hq, d]
+ *   out_f32          optional fp32 copy of out before rounding, same shape
+ *   lse              optional fp32 [B, R, Hq]: natural-log sum of exp of the scaled scores
+ * Math: bf16 operands, fp32 accumulation; softmax weights are rounded to bf16
+ * before multiplying V.  A sequence whose lengths violate the capacity rule is
+ * skipped and MASSV_ERR_CAPACITY is stored in dev_status.
+ */
+int massv_verify_attn(const massv_attn_desc *desc, const void *q, const void *k_new, const void *v_new,
+                      void *k_pages, void *v_pages, const int32_t *page_table, const int32_t *seq_lens,
+                      void *out, float *out_f32, float *lse,
+                      void *workspace, size_t workspace_bytes, int32_t *dev_status, massv_stream_t stream);
+
+/* Bytes of scratch massv_accept needs (0 on a bad descriptor).  Includes room
+ * for the fp32 logits when T > 0, whether or not logits_out is supplied. */
+size_t massv_accept_workspace_size(const massv_accept_desc *desc);
+
+/*
+ * LM head + temperature softmax + speculative acceptance (Sec. 2.1).
+ *
+ * Row (b,j) of `hidden` is the target's final hidden state at block position j;
+ * its logits are z_j = lm_head * hidden[b,j] and, for T > 0, p_j = softmax(z_j / T)
+ * is the target distribution for the token after block position j.
+ *
+ * T > 0: draft j (token x = draft_tokens[b,j], draft distribution
+ *   q_j = draft_probs[b,j,:]) is accepted with probability min(1, p_j(x)/q_j(x)),
+ *   realised with the caller's uniform as  u_accept[b,j] * q_j(x) < p_j(x)
+ *   (fp32).  Drafts are examined in order; at the first rejection n the extra
+ *   token is drawn from norm(max(p_n - q_n, 0)); if all gamma drafts pass
+ *   (n = gamma) it is drawn from p_gamma.  The draw is an inverse-CDF walk in
+ *   vocabulary order with u_sample[b,n]: the first index whose running mass
+ *   exceeds u * total (fp64 running sums); zero-mass tokens are never drawn.
+ *   If the residual has no mass the draw uses p_n.  draft_probs is used as
+ *   given (it is the drafter's distribution at the drafter's temperature).
+ * T == 0: draft j is accepted iff x equals argmax_v z_j[v] (lowest index on
+ *   ties); the extra token is argmax_v z_n[v].  draft_probs, u_accept and
+ *   u_sample are ignored and may be NULL.
+ *
+ *   hidden        bf16 [B, R, K]
+ *   lm_head       bf16 [V, K]
+ *   draft_tokens  int32 [B, gamma], each in [0, V)
+ *   draft_probs   fp32 [B, gamma, V]           (T > 0)
+ *   u_accept      fp32 [B, gamma] in [0,1)     (T > 0)
+ *   u_sample      fp32 [B, R] in [0,1)         (T > 0)
+ *   out_tokens    int32 [B, R]: the n accepted drafts, the extra token, then -1
+ *   accept_len    int32 [B]: n + 1, the tokens gained by this target pass
+ *                 (its batch mean is the paper's mean accepted length tau)
+ *   logits_out    optional fp32 [B, R, V]: z
+ *   probs_out     optional fp32 [B, R, V]: p (T > 0 only; must be NULL at T == 0)
+ * Math: bf16 x bf16 products accumulated in fp32 on the tensor cores.
+ */
+int massv_accept(const massv_accept_desc *desc, const void *hidden, const void *lm_head,
+                 const int32_t *draft_tokens, const float *draft_probs,
+                 const float *u_accept, const float *u_sample,
+                 int32_t *out_tokens, int32_t *accept_len, float *logits_out, float *probs_out,
+                 void *workspace, size_t workspace_bytes, int32_t *dev_status, massv_stream_t stream);
+
+/*
+ * Commit or roll back the speculative block (Sec. 2.1: accepted tokens are
+ * added to the output and the next iteration starts from them).
+ * accept_len != NULL: seq_lens[b] += accept_len[b]; cache rows of block
+ * positions 0 .. n stay, rows beyond are dead and will be overwritten.
+ * accept_len == NULL: rollback, seq_lens is left unchanged, which discards the
+ * whole appended block.  gamma bounds accept_len (values outside [1, gamma+1]
+ * store MASSV_ERR_INVALID_ARG in dev_status and leave that length unchanged).
+ */
+int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t *accept_len, int32_t *seq_lens,
+                    int32_t *dev_status, massv_stream_t stream);
+
+/* Human-readable name of a massv_status value. */
+const char *massv_strerror(int status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int massv_version(void);
+
+/* Number of GPU kernels this library has launched in this process so far
+ * (diagnostic; lets a caller confirm that a call really ran on the device). */
+uint64_t massv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MASSV_H */

@@ -1,0 +1,149 @@
+"""ctypes binding of ``libmassv.so``: argument marshalling only.
+
+Every function takes torch tensors that already live on the GPU (torch is used
+for device memory and streams, nothing else), passes their addresses and the
+current CUDA stream to the C entry point of the same name, and raises
+``MassvError`` on a non-zero status.  There is no CPU path: importing this
+module without the compiled library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmassv.so")
+
+
+class MassvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {_strerror(status)} (status {status})")
+
+
+class AttnDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("gamma", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
+                ("max_pages_per_seq", ctypes.c_int32), ("num_pages", ctypes.c_int64), ("scale", ctypes.c_float),
+                ("kv_chunk", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class AcceptDesc(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("gamma", ctypes.c_int32), ("hidden", ctypes.c_int32),
+                ("vocab", ctypes.c_int32), ("temperature", ctypes.c_float), ("flags", ctypes.c_uint32)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2505_10526_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+    lib.massv_verify_attn_workspace_size.restype = ctypes.c_size_t
+    lib.massv_verify_attn_workspace_size.argtypes = [ctypes.POINTER(AttnDesc)]
+    lib.massv_verify_attn.restype = ctypes.c_int
+    lib.massv_verify_attn.argtypes = [ctypes.POINTER(AttnDesc), vp, vp, vp, vp, vp, i32p, i32p, vp, f32p, f32p,
+                                      vp, ctypes.c_size_t, i32p, vp]
+    lib.massv_accept_workspace_size.restype = ctypes.c_size_t
+    lib.massv_accept_workspace_size.argtypes = [ctypes.POINTER(AcceptDesc)]
+    lib.massv_accept.restype = ctypes.c_int
+    lib.massv_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, i32p, f32p, f32p, f32p, i32p, i32p, f32p, f32p,
+                                 vp, ctypes.c_size_t, i32p, vp]
+    lib.massv_kv_commit.restype = ctypes.c_int
+    lib.massv_kv_commit.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, vp]
+    lib.massv_strerror.restype = ctypes.c_char_p
+    lib.massv_strerror.argtypes = [ctypes.c_int]
+    lib.massv_version.restype = ctypes.c_int
+    lib.massv_launch_count.restype = ctypes.c_uint64
+    return lib
+
+
+_lib = _load()
+
+
+def _strerror(status: int) -> str:
+    return _lib.massv_strerror(int(status)).decode()
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("massv: tensors must live on a CUDA device")
+    if not t.is_contiguous():
+        raise ValueError("massv: tensors must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"massv: expected {dtype}, got {t.dtype}")
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def massv_version() -> int:
+    return int(_lib.massv_version())
+
+
+def massv_launch_count() -> int:
+    return int(_lib.massv_launch_count())
+
+
+def massv_strerror(status: int) -> str:
+    return _strerror(status)
+
+
+def attn_desc(batch, gamma, n_q_heads, n_kv_heads, head_dim, max_pages_per_seq, num_pages, scale=0.0, kv_chunk=0,
+              page_size=16) -> AttnDesc:
+    return AttnDesc(batch, gamma, n_q_heads, n_kv_heads, head_dim, page_size, max_pages_per_seq, num_pages,
+                    float(scale), kv_chunk, 0)
+
+
+def accept_desc(batch, gamma, hidden, vocab, temperature) -> AcceptDesc:
+    return AcceptDesc(batch, gamma, hidden, vocab, float(temperature), 0)
+
+
+def massv_verify_attn_workspace_size(desc: AttnDesc) -> int:
+    return int(_lib.massv_verify_attn_workspace_size(ctypes.byref(desc)))
+
+
+def massv_accept_workspace_size(desc: AcceptDesc) -> int:
+    return int(_lib.massv_accept_workspace_size(ctypes.byref(desc)))
+
+
+def alloc_workspace(nbytes: int, device) -> torch.Tensor:
+    """A 256-byte aligned scratch buffer (torch's caching allocator aligns to 512)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def massv_verify_attn(desc, q, k_new, v_new, k_pages, v_pages, page_table, seq_lens, out, out_f32=None, lse=None,
+                      workspace=None, dev_status=None) -> None:
+    bf = torch.bfloat16
+    rc = _lib.massv_verify_attn(ctypes.byref(desc), _ptr(q, bf), _ptr(k_new, bf), _ptr(v_new, bf), _ptr(k_pages, bf),
+                                _ptr(v_pages, bf), _ptr(page_table, torch.int32), _ptr(seq_lens, torch.int32),
+                                _ptr(out, bf), _ptr(out_f32, torch.float32), _ptr(lse, torch.float32),
+                                _ptr(workspace), workspace.numel() if workspace is not None else 0,
+                                _ptr(dev_status, torch.int32), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_verify_attn")
+
+
+def massv_accept(desc, hidden, lm_head, draft_tokens, draft_probs, u_accept, u_sample, out_tokens, accept_len,
+                 logits_out=None, probs_out=None, workspace=None, dev_status=None) -> None:
+    bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
+    rc = _lib.massv_accept(ctypes.byref(desc), _ptr(hidden, bf), _ptr(lm_head, bf), _ptr(draft_tokens, i32),
+                           _ptr(draft_probs, f32), _ptr(u_accept, f32), _ptr(u_sample, f32), _ptr(out_tokens, i32),
+                           _ptr(accept_len, i32), _ptr(logits_out, f32), _ptr(probs_out, f32),
+                           _ptr(workspace), workspace.numel() if workspace is not None else 0,
+                           _ptr(dev_status, i32), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_accept")
+
+
+def massv_kv_commit(batch, gamma, accept_len, seq_lens, dev_status=None) -> None:
+    rc = _lib.massv_kv_commit(batch, gamma, _ptr(accept_len, torch.int32), _ptr(seq_lens, torch.int32),
+                              _ptr(dev_status, torch.int32), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_kv_commit")

@@ -1,0 +1,315 @@
+// Speculative acceptance after the LM head (paper Sec. 2.1):
+//   accept_scan_kernel      reduces the per-tile softmax statistics of every block
+//                           row, runs the sequential accept/reject scan, and at
+//                           T == 0 also emits the extra token (the row's argmax);
+//   residual_sample_kernel  T > 0: one vocabulary pass over the single row the
+//                           extra token is drawn from (residual max(p-q,0) after
+//                           a rejection, p itself for the bonus token), as chunk
+//                           masses followed by an inverse-CDF walk in fp64;
+//   probs_kernel            optional dense p = softmax(z/T) output;
+//   kv_commit_kernel        advance the committed cache lengths.
+// All reductions run in a fixed order, so results are bit-identical run to run.
+#include "kernels.cuh"
+
+namespace massv {
+
+namespace {
+
+constexpr int kScanThreads = 256;
+constexpr int kSampleThreads = 256;
+constexpr int kPerThread = kResidualChunk / kSampleThreads;   // 16 contiguous entries per thread
+static_assert(kPerThread == 16, "chunk layout");
+
+struct Stat {
+    float m;   // running max logit
+    float s;   // sum of exp((z - m)/T)
+    int idx;   // lowest index attaining m
+};
+
+__device__ __forceinline__ Stat combine(Stat a, Stat b, float inv_T) {
+    if (b.m == -INFINITY) return a;
+    if (a.m == -INFINITY) return b;
+    Stat r;
+    r.m = fmaxf(a.m, b.m);
+    r.s = a.s * expf((a.m - r.m) * inv_T) + b.s * expf((b.m - r.m) * inv_T);
+    r.idx = (a.m > b.m || (a.m == b.m && a.idx < b.idx)) ? a.idx : b.idx;
+    return r;
+}
+
+// One CTA per sequence.
+__global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams p) {
+    const int b = blockIdx.x, t = threadIdx.x;
+    const int R = p.gamma + 1, M = p.B * R;
+    const bool greedy = !(p.T > 0.f);
+    const float inv_T = greedy ? 1.f : 1.f / p.T;
+    __shared__ Stat red[kScanThreads];
+    __shared__ Stat row_stat[kMaxRows];
+
+    for (int j = 0; j < R; ++j) {
+        const int row = b * R + j;
+        Stat acc{-INFINITY, 0.f, 0x7fffffff};
+        for (int i = t; i < p.n_part; i += kScanThreads) {
+            Stat x{p.part_max[(size_t)i * M + row], greedy ? 0.f : p.part_sum[(size_t)i * M + row],
+                   p.part_idx[(size_t)i * M + row]};
+            acc = combine(acc, x, inv_T);
+        }
+        red[t] = acc;
+        __syncthreads();
+        for (int w = kScanThreads / 2; w > 0; w >>= 1) {
+            if (t < w) red[t] = combine(red[t], red[t + w], inv_T);
+            __syncthreads();
+        }
+        if (t == 0) row_stat[j] = red[0];
+        __syncthreads();
+    }
+    if (t != 0) return;
+
+    int n = p.gamma;
+    int32_t* toks = p.out_tokens + (size_t)b * R;
+    for (int j = 0; j < R; ++j) toks[j] = -1;
+    for (int j = 0; j < p.gamma; ++j) {
+        const int x = p.draft_tokens[(size_t)b * p.gamma + j];
+        bool ok;
+        if (x < 0 || x >= p.V) {
+            set_status(p.dev_status, MASSV_ERR_INVALID_ARG);
+            ok = false;
+        } else if (greedy) {
+            ok = (x == row_stat[j].idx);
+        } else {
+            const float zx = p.logits[(size_t)(b * R + j) * p.V + x];
+            const float px = expf((zx - row_stat[j].m) * inv_T) / row_stat[j].s;
+            const float qx = p.draft_probs[((size_t)b * p.gamma + j) * p.V + x];
+            const float lhs = p.u_accept[(size_t)b * p.gamma + j] * qx;
+            ok = lhs < px;
+        }
+        if (!ok) { n = j; break; }
+        toks[j] = x;
+    }
+    p.accept_len[b] = n + 1;
+    if (greedy) {
+        toks[n] = row_stat[n].idx;
+    } else {
+        SeqState st;
+        st.n = n;
+        st.use_q = n < p.gamma ? 1 : 0;
+        st.row_max = row_stat[n].m;
+        st.inv_sum = 1.f / row_stat[n].s;
+        p.seq_state[b] = st;
+        p.counters[b] = 0u;
+    }
+}
+
+// Masses of the 16 entries this thread owns in chunk c of the sampled row.
+__device__ __forceinline__ void chunk_masses(const AcceptParams& p, int b, const SeqState& st, int use_q, int c,
+                                             float inv_T, float (&r)[kPerThread]) {
+    const int R = p.gamma + 1;
+    const int v0 = c * kResidualChunk + threadIdx.x * kPerThread;
+    const float* z = p.logits + (size_t)(b * R + st.n) * p.V;
+    const float* q = use_q ? p.draft_probs + ((size_t)b * p.gamma + st.n) * p.V : nullptr;
+#pragma unroll
+    for (int g = 0; g < kPerThread; g += 4) {
+        const int v = v0 + g;
+        float zz[4] = {0.f, 0.f, 0.f, 0.f}, qq[4] = {0.f, 0.f, 0.f, 0.f};
+        if (v + 3 < p.V) {
+            const float4 a = *reinterpret_cast<const float4*>(z + v);
+            zz[0] = a.x; zz[1] = a.y; zz[2] = a.z; zz[3] = a.w;
+            if (q) {
+                const float4 d = __ldg(reinterpret_cast<const float4*>(q + v));
+                qq[0] = d.x; qq[1] = d.y; qq[2] = d.z; qq[3] = d.w;
+            }
+        } else {
+            for (int e = 0; e < 4; ++e)
+                if (v + e < p.V) { zz[e] = z[v + e]; if (q) qq[e] = q[v + e]; }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float m = 0.f;
+            if (v + e < p.V) {
+                const float pv = expf((zz[e] - st.row_max) * inv_T) * st.inv_sum;
+                m = q ? fmaxf(pv - qq[e], 0.f) : pv;
+            }
+            r[g + e] = m;
+        }
+    }
+}
+
+// Block-wide exclusive prefix of one double per thread, in thread order; *total gets the sum.
+__device__ __forceinline__ double block_exclusive_scan(double x, double* smem_warp, double* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    double incl = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    if (lane == 31) smem_warp[warp] = incl;
+    __syncthreads();
+    double base = 0.0, tot = 0.0;
+    for (int w = 0; w < kSampleThreads / 32; ++w) {
+        const double s = smem_warp[w];
+        if (w < warp) base += s;
+        tot += s;
+    }
+    __syncthreads();
+    *total = tot;
+    return base + incl - x;
+}
+
+// grid (n_chunks, B).  Every CTA stores its chunk's mass; the CTA that arrives
+// last for a sequence walks the chunk masses and then the winning chunk.
+__global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptParams p) {
+    const int c = blockIdx.x, b = blockIdx.y, t = threadIdx.x;
+    const int R = p.gamma + 1;
+    const float inv_T = 1.f / p.T;
+    const SeqState st = p.seq_state[b];
+    __shared__ double warp_sums[kSampleThreads / 32];
+    __shared__ int s_flag;
+    __shared__ int s_pick[2];
+    __shared__ double s_base[2];
+
+    float r[kPerThread];
+    chunk_masses(p, b, st, st.use_q, c, inv_T, r);
+    double local = 0.0;
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) local += (double)r[e];
+    double total;
+    block_exclusive_scan(local, warp_sums, &total);
+    double* sums = p.chunk_sums + (size_t)b * p.n_chunks;
+    if (t == 0) {
+        sums[c] = total;
+        __threadfence();
+        const unsigned prev = atomicAdd(&p.counters[b], 1u);
+        s_flag = (prev == (unsigned)p.n_chunks - 1u);
+    }
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+
+    int use_q = st.use_q;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        // sequential walk over the chunk masses (a few dozen doubles)
+        if (t == 0) {
+            double tot = 0.0;
+            for (int i = 0; i < p.n_chunks; ++i) tot += ((volatile double*)sums)[i];
+            const double target = (double)p.u_sample[(size_t)b * R + st.n] * tot;
+            int pick = -1, last_pos = -1;
+            double cum = 0.0, base = 0.0;
+            for (int i = 0; i < p.n_chunks; ++i) {
+                const double s = ((volatile double*)sums)[i];
+                if (s > 0.0) last_pos = i;
+                if (pick < 0 && s > 0.0 && cum + s > target) { pick = i; base = cum; }
+                cum += s;
+            }
+            s_pick[0] = tot > 0.0 ? (pick >= 0 ? pick : last_pos) : -1;
+            s_pick[1] = (pick < 0);        // rounding pushed the target past the end: take the last positive entry
+            s_base[0] = base;
+            s_base[1] = target;
+        }
+        __syncthreads();
+        if (s_pick[0] >= 0 || !use_q) break;
+        // The residual has no mass (p == q on this row): draw from p instead.
+        use_q = 0;
+        for (int cc = 0; cc < p.n_chunks; ++cc) {
+            chunk_masses(p, b, st, 0, cc, inv_T, r);
+            double loc = 0.0;
+#pragma unroll
+            for (int e = 0; e < kPerThread; ++e) loc += (double)r[e];
+            double tt;
+            block_exclusive_scan(loc, warp_sums, &tt);
+            if (t == 0) sums[cc] = tt;
+        }
+        __syncthreads();
+    }
+    const int pick = s_pick[0];
+    int32_t* tok_out = p.out_tokens + (size_t)b * R + st.n;
+    if (pick < 0) {                        // no mass at all (cannot happen for a softmax row)
+        if (t == 0) { *tok_out = 0; set_status(p.dev_status, MASSV_ERR_INVALID_ARG); }
+        return;
+    }
+    const bool take_last = s_pick[1] != 0;
+    const double base = s_base[0], target = s_base[1];
+    chunk_masses(p, b, st, use_q, pick, inv_T, r);
+    double loc = 0.0;
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) loc += (double)r[e];
+    double tt;
+    double run = base + block_exclusive_scan(loc, warp_sums, &tt);
+    int first = 0x7fffffff, last = -1;
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) {
+        run += (double)r[e];
+        if (r[e] > 0.f) {
+            const int v = pick * kResidualChunk + t * kPerThread + e;
+            last = v;
+            if (first == 0x7fffffff && run > target) first = v;
+        }
+    }
+    __shared__ int s_first, s_last;
+    if (t == 0) { s_first = 0x7fffffff; s_last = -1; }
+    __syncthreads();
+    atomicMin(&s_first, first);
+    atomicMax(&s_last, last);
+    __syncthreads();
+    if (t == 0) *tok_out = (!take_last && s_first != 0x7fffffff) ? s_first : s_last;
+}
+
+// Dense probabilities for callers that ask for them (diagnostics / tests).
+__global__ void probs_kernel(AcceptParams p) {
+    const int R = p.gamma + 1, M = p.B * R;
+    const int row = blockIdx.y;
+    if (row >= M) return;
+    const float inv_T = 1.f / p.T;
+    __shared__ Stat red[256];
+    __shared__ Stat rs;
+    Stat acc{-INFINITY, 0.f, 0x7fffffff};
+    for (int i = threadIdx.x; i < p.n_part; i += blockDim.x) {
+        Stat x{p.part_max[(size_t)i * M + row], p.part_sum[(size_t)i * M + row], p.part_idx[(size_t)i * M + row]};
+        acc = combine(acc, x, inv_T);
+    }
+    red[threadIdx.x] = acc;
+    __syncthreads();
+    for (int w = blockDim.x / 2; w > 0; w >>= 1) {
+        if (threadIdx.x < w) red[threadIdx.x] = combine(red[threadIdx.x], red[threadIdx.x + w], inv_T);
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) rs = red[0];
+    __syncthreads();
+    const float inv_sum = 1.f / rs.s;
+    for (int v = blockIdx.x * blockDim.x + threadIdx.x; v < p.V; v += gridDim.x * blockDim.x)
+        p.probs_out[(size_t)row * p.V + v] = expf((p.logits[(size_t)row * p.V + v] - rs.m) * inv_T) * inv_sum;
+}
+
+__global__ void kv_commit_kernel(int B, int gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int a = accept_len[b];
+    if (a < 1 || a > gamma + 1) { set_status(dev_status, MASSV_ERR_INVALID_ARG); return; }
+    seq_lens[b] += a;
+}
+
+}  // namespace
+
+cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream) {
+    accept_scan_kernel<<<p.B, kScanThreads, 0, stream>>>(p);
+    count_launches(1);
+    if (p.T > 0.f) {
+        residual_sample_kernel<<<dim3(p.n_chunks, p.B), kSampleThreads, 0, stream>>>(p);
+        count_launches(1);
+        if (p.probs_out) {
+            const int M = p.B * (p.gamma + 1);
+            probs_kernel<<<dim3(16, M), 256, 0, stream>>>(p);
+            count_launches(1);
+        }
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_kv_commit(int B, int gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
+                             cudaStream_t stream) {
+    if (accept_len == nullptr) return cudaSuccess;   // rollback: lengths stay
+    kv_commit_kernel<<<(B + 127) / 128, 128, 0, stream>>>(B, gamma, accept_len, seq_lens, dev_status);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace massv

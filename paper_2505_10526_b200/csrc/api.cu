@@ -1,0 +1,221 @@
+// C ABI of the verify-step library: host-side validation, workspace layout and
+// kernel launches.  No device memory is allocated and no stream is synchronised.
+#include <math.h>
+
+#include <atomic>
+
+#include "kernels.cuh"
+
+using namespace massv;
+
+static std::atomic<uint64_t> g_launches{0};
+namespace massv {
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+}
+
+namespace {
+
+constexpr size_t kAlign = 256;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int auto_kv_chunk(const massv_attn_desc& d) {
+    // Aim at roughly four resident work items per SM over the longest context
+    // the page table can describe; never split finer than 64 tokens.
+    const double tokens = (double)d.batch * d.max_pages_per_seq * kPageSize * d.n_kv_heads;
+    long chunk = (long)ceil(tokens / (148.0 * 4.0));
+    chunk = (chunk + 63) / 64 * 64;
+    if (chunk < 64) chunk = 64;
+    if (chunk > 4096) chunk = 4096;
+    return (int)chunk;
+}
+
+int check_attn_desc(const massv_attn_desc* d) {
+    if (!d) return MASSV_ERR_INVALID_ARG;
+    if (d->batch < 1 || d->n_q_heads < 1 || d->n_kv_heads < 1 || d->max_pages_per_seq < 1 || d->num_pages < 1 ||
+        d->gamma < 0 || d->scale < 0.f || d->kv_chunk < 0)
+        return MASSV_ERR_INVALID_ARG;
+    if (d->gamma > kMaxRows - 1) return MASSV_ERR_UNSUPPORTED;
+    if (d->page_size != kPageSize) return MASSV_ERR_UNSUPPORTED;
+    if (d->head_dim != 64 && d->head_dim != 128 && d->head_dim != 256) return MASSV_ERR_UNSUPPORTED;
+    if (d->n_q_heads % d->n_kv_heads != 0) return MASSV_ERR_UNSUPPORTED;
+    if ((d->n_q_heads / d->n_kv_heads) * (d->gamma + 1) > 64) return MASSV_ERR_UNSUPPORTED;
+    if (d->kv_chunk % 64 != 0) return MASSV_ERR_UNSUPPORTED;
+    if (d->flags != 0) return MASSV_ERR_UNSUPPORTED;
+    return MASSV_OK;
+}
+
+struct AttnLayout {
+    int kv_chunk, max_chunks, rows_pad;
+    size_t off_o, off_ml, total;
+};
+
+AttnLayout attn_layout(const massv_attn_desc& d) {
+    AttnLayout l;
+    l.kv_chunk = d.kv_chunk > 0 ? d.kv_chunk : auto_kv_chunk(d);
+    const long max_tokens = (long)d.max_pages_per_seq * kPageSize;
+    l.max_chunks = (int)((max_tokens + l.kv_chunk - 1) / l.kv_chunk);
+    l.rows_pad = attn_rows_pad((d.n_q_heads / d.n_kv_heads) * (d.gamma + 1));
+    const size_t items = (size_t)d.batch * d.n_kv_heads * l.max_chunks;
+    l.off_o = 0;
+    l.off_ml = align_up(items * l.rows_pad * d.head_dim * sizeof(float), kAlign);
+    l.total = l.off_ml + align_up(items * l.rows_pad * 2 * sizeof(float), kAlign);
+    return l;
+}
+
+int check_accept_desc(const massv_accept_desc* d) {
+    if (!d) return MASSV_ERR_INVALID_ARG;
+    if (d->batch < 1 || d->gamma < 0 || d->hidden < 1 || d->vocab < 1 || !(d->temperature >= 0.f))
+        return MASSV_ERR_INVALID_ARG;
+    if (d->gamma > kMaxRows - 1) return MASSV_ERR_UNSUPPORTED;
+    if ((long)d->batch * (d->gamma + 1) > 512) return MASSV_ERR_UNSUPPORTED;
+    if (d->hidden % 64 != 0 || d->vocab % 8 != 0) return MASSV_ERR_UNSUPPORTED;
+    if (d->flags != 0) return MASSV_ERR_UNSUPPORTED;
+    return MASSV_OK;
+}
+
+struct AcceptLayout {
+    int n_part, n_chunks;
+    size_t off_max, off_sum, off_idx, off_state, off_chunks, off_counters, off_logits, total;
+};
+
+AcceptLayout accept_layout(const massv_accept_desc& d) {
+    AcceptLayout l;
+    const size_t M = (size_t)d.batch * (d.gamma + 1);
+    l.n_part = lm_head_num_partials((int)M, d.vocab);
+    l.n_chunks = (d.vocab + kResidualChunk - 1) / kResidualChunk;
+    size_t off = 0;
+    l.off_max = off; off += align_up((size_t)l.n_part * M * sizeof(float), kAlign);
+    l.off_sum = off; off += align_up((size_t)l.n_part * M * sizeof(float), kAlign);
+    l.off_idx = off; off += align_up((size_t)l.n_part * M * sizeof(int32_t), kAlign);
+    l.off_state = off; off += align_up((size_t)d.batch * sizeof(SeqState), kAlign);
+    l.off_chunks = off; off += align_up((size_t)d.batch * l.n_chunks * sizeof(double), kAlign);
+    l.off_counters = off; off += align_up((size_t)d.batch * sizeof(unsigned int), kAlign);
+    l.off_logits = off; off += align_up(M * (size_t)d.vocab * sizeof(float), kAlign);
+    l.total = off;
+    return l;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t massv_verify_attn_workspace_size(const massv_attn_desc* desc) {
+    if (check_attn_desc(desc) != MASSV_OK) return 0;
+    return attn_layout(*desc).total;
+}
+
+int massv_verify_attn(const massv_attn_desc* desc, const void* q, const void* k_new, const void* v_new,
+                      void* k_pages, void* v_pages, const int32_t* page_table, const int32_t* seq_lens,
+                      void* out, float* out_f32, float* lse, void* workspace, size_t workspace_bytes,
+                      int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_attn_desc(desc);
+    if (rc != MASSV_OK) return rc;
+    if (!q || !k_new || !v_new || !k_pages || !v_pages || !page_table || !seq_lens || !out) return MASSV_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(k_pages) || !aligned16(v_pages) ||
+        !aligned16(out) || (out_f32 && !aligned16(out_f32)))
+        return MASSV_ERR_INVALID_ARG;
+    const AttnLayout l = attn_layout(*desc);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0 || workspace_bytes < l.total)
+        return MASSV_ERR_WORKSPACE;
+
+    AttnParams p;
+    p.B = desc->batch; p.R = desc->gamma + 1; p.Hq = desc->n_q_heads; p.Hkv = desc->n_kv_heads;
+    p.d = desc->head_dim; p.max_pages = desc->max_pages_per_seq; p.num_pages = desc->num_pages;
+    p.scale = desc->scale > 0.f ? desc->scale : 1.f / sqrtf((float)desc->head_dim);
+    p.kv_chunk = l.kv_chunk; p.max_chunks = l.max_chunks;
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+    p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+    p.k_pages = static_cast<__nv_bfloat16*>(k_pages);
+    p.v_pages = static_cast<__nv_bfloat16*>(v_pages);
+    p.page_table = page_table; p.seq_lens = seq_lens;
+    p.out = static_cast<__nv_bfloat16*>(out); p.out_f32 = out_f32; p.lse = lse;
+    char* ws = static_cast<char*>(workspace);
+    p.part_o = reinterpret_cast<float*>(ws + l.off_o);
+    p.part_ml = reinterpret_cast<float*>(ws + l.off_ml);
+    p.dev_status = dev_status;
+    return launch_verify_attn(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
+size_t massv_accept_workspace_size(const massv_accept_desc* desc) {
+    if (check_accept_desc(desc) != MASSV_OK) return 0;
+    return accept_layout(*desc).total;
+}
+
+int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* lm_head, const int32_t* draft_tokens,
+                 const float* draft_probs, const float* u_accept, const float* u_sample, int32_t* out_tokens,
+                 int32_t* accept_len, float* logits_out, float* probs_out, void* workspace, size_t workspace_bytes,
+                 int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_accept_desc(desc);
+    if (rc != MASSV_OK) return rc;
+    const bool sampling = desc->temperature > 0.f;
+    if (!hidden || !lm_head || !out_tokens || !accept_len) return MASSV_ERR_INVALID_ARG;
+    if (desc->gamma > 0 && !draft_tokens) return MASSV_ERR_INVALID_ARG;
+    if (sampling && (!u_sample || (desc->gamma > 0 && (!draft_probs || !u_accept)))) return MASSV_ERR_INVALID_ARG;
+    if (!sampling && probs_out) return MASSV_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(lm_head) || (draft_probs && !aligned16(draft_probs)) ||
+        (logits_out && !aligned16(logits_out)) || (probs_out && !aligned16(probs_out)))
+        return MASSV_ERR_INVALID_ARG;
+    const AcceptLayout l = accept_layout(*desc);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0 || workspace_bytes < l.total)
+        return MASSV_ERR_WORKSPACE;
+    char* ws = static_cast<char*>(workspace);
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+
+    LmHeadParams g;
+    g.M = desc->batch * (desc->gamma + 1); g.K = desc->hidden; g.V = desc->vocab;
+    g.greedy = sampling ? 0 : 1;
+    g.inv_T_log2e = sampling ? 1.4426950408889634f / desc->temperature : 0.f;
+    g.hidden = static_cast<const __nv_bfloat16*>(hidden);
+    g.lm_head = static_cast<const __nv_bfloat16*>(lm_head);
+    g.logits = logits_out ? logits_out : reinterpret_cast<float*>(ws + l.off_logits);
+    g.n_part = l.n_part;
+    g.part_max = reinterpret_cast<float*>(ws + l.off_max);
+    g.part_sum = reinterpret_cast<float*>(ws + l.off_sum);
+    g.part_idx = reinterpret_cast<int32_t*>(ws + l.off_idx);
+    g.dev_status = dev_status;
+    if (launch_lm_head(g, s) != cudaSuccess) return MASSV_ERR_CUDA;
+
+    AcceptParams a;
+    a.B = desc->batch; a.gamma = desc->gamma; a.V = desc->vocab; a.T = desc->temperature;
+    a.n_part = l.n_part; a.part_max = g.part_max; a.part_sum = g.part_sum; a.part_idx = g.part_idx;
+    a.logits = g.logits;
+    a.draft_tokens = draft_tokens; a.draft_probs = draft_probs; a.u_accept = u_accept; a.u_sample = u_sample;
+    a.out_tokens = out_tokens; a.accept_len = accept_len; a.probs_out = probs_out;
+    a.seq_state = reinterpret_cast<SeqState*>(ws + l.off_state);
+    a.chunk_sums = reinterpret_cast<double*>(ws + l.off_chunks);
+    a.counters = reinterpret_cast<unsigned int*>(ws + l.off_counters);
+    a.n_chunks = l.n_chunks;
+    a.dev_status = dev_status;
+    return launch_accept(a, s) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
+int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
+                    massv_stream_t stream) {
+    if (batch < 1 || gamma < 0 || !seq_lens) return MASSV_ERR_INVALID_ARG;
+    if (gamma > kMaxRows - 1) return MASSV_ERR_UNSUPPORTED;
+    return launch_kv_commit(batch, gamma, accept_len, seq_lens, dev_status, reinterpret_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess
+               ? MASSV_OK
+               : MASSV_ERR_CUDA;
+}
+
+const char* massv_strerror(int status) {
+    switch (status) {
+        case MASSV_OK: return "ok";
+        case MASSV_ERR_INVALID_ARG: return "invalid argument";
+        case MASSV_ERR_UNSUPPORTED: return "unsupported shape";
+        case MASSV_ERR_CAPACITY: return "page table capacity exceeded or unmapped page";
+        case MASSV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case MASSV_ERR_CUDA: return "CUDA call failed";
+        case MASSV_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+int massv_version(void) { return 100; }
+
+uint64_t massv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,65 @@
+// Internal launch interfaces between the C ABI (api.cu) and the kernels.
+#pragma once
+
+#include "common.cuh"
+
+namespace massv {
+
+// ---------------------------------------------------------------- attention
+struct AttnParams {
+    int B, R, Hq, Hkv, d, max_pages;
+    int64_t num_pages;
+    float scale;
+    int kv_chunk;      // tokens per split
+    int max_chunks;    // splits launched per (sequence, kv head)
+    const __nv_bfloat16 *q, *k_new, *v_new;
+    __nv_bfloat16 *k_pages, *v_pages;
+    const int32_t *page_table, *seq_lens;
+    __nv_bfloat16* out;
+    float *out_f32, *lse;
+    float* part_o;     // [B, Hkv, max_chunks, rows_pad, d] unnormalised partial outputs
+    float* part_ml;    // [B, Hkv, max_chunks, rows_pad, 2] running max (log2 domain) and sum
+    int32_t* dev_status;
+};
+int attn_rows_pad(int group_rows);                 // query rows per KV head, padded to the MMA tile
+cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream);
+
+// ---------------------------------------------------------------- LM head
+struct LmHeadParams {
+    int M, K, V;
+    float inv_T_log2e;              // log2(e)/T; unused at T == 0
+    int greedy;                     // 1: T == 0 (no sum of exponentials, no logits needed)
+    const __nv_bfloat16 *hidden, *lm_head;
+    float* logits;                  // [M, V] or nullptr
+    int n_part;                     // partial slots available
+    float *part_max, *part_sum;     // [n_part, M]
+    int32_t* part_idx;              // [n_part, M]
+    int32_t* dev_status;
+};
+int lm_head_num_partials(int M, int V);            // slots the kernel fills for this shape
+cudaError_t launch_lm_head(const LmHeadParams& p, cudaStream_t stream);
+
+// ---------------------------------------------------------------- acceptance
+struct AcceptParams {
+    int B, gamma, V;
+    float T;
+    int n_part;
+    const float *part_max, *part_sum;
+    const int32_t* part_idx;
+    const float* logits;            // [B*(gamma+1), V], T > 0 only
+    const int32_t* draft_tokens;
+    const float *draft_probs, *u_accept, *u_sample;
+    int32_t *out_tokens, *accept_len;
+    float* probs_out;               // optional
+    SeqState* seq_state;            // [B]
+    double* chunk_sums;             // [B, n_chunks]
+    unsigned int* counters;         // [B]
+    int n_chunks;
+    int32_t* dev_status;
+};
+cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream);
+
+cudaError_t launch_kv_commit(int B, int gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
+                             cudaStream_t stream);
+
+}  // namespace massv

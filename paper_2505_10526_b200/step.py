@@ -1,0 +1,94 @@
+"""One verify step = massv_verify_attn + massv_accept + massv_kv_commit.
+
+``VerifyStep`` owns the descriptors, the scratch buffers and the output tensors
+for a fixed geometry, so that a step is three C-ABI calls and nothing else.  All
+arithmetic happens inside ``libmassv.so``.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as mv
+
+# tensors that change every step (the rest - page pools, page table, lengths,
+# LM-head weights - is resident state)
+STEP_INPUTS = ("q", "k_new", "v_new", "hidden", "draft_tokens", "draft_probs", "u_accept", "u_sample")
+
+
+class VerifyStep:
+    def __init__(self, batch, gamma, n_q_heads, n_kv_heads, head_dim, hidden, vocab, temperature,
+                 max_pages_per_seq, num_pages, device="cuda", kv_chunk=0, scale=0.0,
+                 want_logits=False, want_probs=False, want_attn_f32=False):
+        self.device = torch.device(device)
+        self.B, self.gamma, self.R = batch, gamma, gamma + 1
+        self.T = float(temperature)
+        self.adesc = mv.attn_desc(batch, gamma, n_q_heads, n_kv_heads, head_dim, max_pages_per_seq, num_pages,
+                                  scale=scale, kv_chunk=kv_chunk)
+        self.cdesc = mv.accept_desc(batch, gamma, hidden, vocab, temperature)
+        dev = self.device
+        self.attn_ws = mv.alloc_workspace(mv.massv_verify_attn_workspace_size(self.adesc), dev)
+        self.accept_ws = mv.alloc_workspace(mv.massv_accept_workspace_size(self.cdesc), dev)
+        self.attn_out = torch.empty((batch, self.R, n_q_heads, head_dim), dtype=torch.bfloat16, device=dev)
+        self.attn_out_f32 = torch.empty_like(self.attn_out, dtype=torch.float32) if want_attn_f32 else None
+        self.lse = torch.empty((batch, self.R, n_q_heads), dtype=torch.float32, device=dev) if want_attn_f32 else None
+        self.out_tokens = torch.empty((batch, self.R), dtype=torch.int32, device=dev)
+        self.accept_len = torch.empty((batch,), dtype=torch.int32, device=dev)
+        self.logits = torch.empty((batch, self.R, vocab), dtype=torch.float32, device=dev) if want_logits else None
+        self.probs = (torch.empty((batch, self.R, vocab), dtype=torch.float32, device=dev)
+                      if want_probs and temperature > 0 else None)
+        self.dev_status = torch.zeros((1,), dtype=torch.int32, device=dev)
+        self._staging = None
+        self._host_out = None
+
+    @classmethod
+    def for_workload(cls, cfg, w, **kw):
+        return cls(cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.hidden, cfg.vocab,
+                   cfg.temperature, w["page_table"].shape[1], w["k_pages"].shape[0],
+                   device=w["k_pages"].device, **kw)
+
+    # -- the three calls -------------------------------------------------------------
+    def attn(self, w):
+        mv.massv_verify_attn(self.adesc, w["q"], w["k_new"], w["v_new"], w["k_pages"], w["v_pages"],
+                             w["page_table"], w["seq_lens"], self.attn_out, self.attn_out_f32, self.lse,
+                             self.attn_ws, self.dev_status)
+
+    def accept(self, w):
+        sampling = self.T > 0
+        mv.massv_accept(self.cdesc, w["hidden"], w["lm_head"], w["draft_tokens"],
+                        w.get("draft_probs") if sampling else None, w.get("u_accept") if sampling else None,
+                        w.get("u_sample") if sampling else None, self.out_tokens, self.accept_len,
+                        self.logits, self.probs, self.accept_ws, self.dev_status)
+
+    def commit(self, seq_lens, rollback=False):
+        mv.massv_kv_commit(self.B, self.gamma, None if rollback else self.accept_len, seq_lens, self.dev_status)
+
+    def run(self, w, commit=True):
+        """Enqueue one whole step on the current stream (no synchronisation)."""
+        self.attn(w)
+        self.accept(w)
+        if commit:
+            self.commit(w["seq_lens"])
+
+    # -- end-to-end step with host buffers ----------------------------------------------
+    def run_host(self, host_inputs, resident, commit=False):
+        """One step whose per-step inputs start in pinned host memory and whose
+        result (tokens and accepted lengths) ends in pinned host memory.
+        Returns (out_tokens, accept_len) host tensors after synchronising."""
+        if self._staging is None:
+            self._staging = {k: torch.empty_like(v, device=self.device) for k, v in host_inputs.items()}
+            self._host_out = (torch.empty(self.out_tokens.shape, dtype=torch.int32).pin_memory(),
+                              torch.empty(self.accept_len.shape, dtype=torch.int32).pin_memory())
+        w = dict(resident)
+        for k, v in host_inputs.items():
+            self._staging[k].copy_(v, non_blocking=True)
+            w[k] = self._staging[k]
+        self.run(w, commit=commit)
+        self._host_out[0].copy_(self.out_tokens, non_blocking=True)
+        self._host_out[1].copy_(self.accept_len, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return self._host_out
+
+    def host_bytes_per_step(self, host_inputs):
+        h2d = sum(v.numel() * v.element_size() for v in host_inputs.values())
+        d2h = self.out_tokens.numel() * 4 + self.accept_len.numel() * 4
+        return h2d, d2h

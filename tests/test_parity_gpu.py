@@ -1,0 +1,192 @@
+"""CUDA path vs CPU oracle, element by element, through the C ABI.
+
+Tolerances (absolute): logits 2e-2 (bf16 operands, fp32 accumulation),
+probabilities 1e-4, attention output 2e-2 in bf16 / 5e-3 in fp32 (softmax
+weights are rounded to bf16 before the PV product), log-sum-exp 1e-3.
+Integer outputs (appended cache bytes, tokens, accepted lengths, committed
+lengths) are bit-exact except at decisions whose oracle margin is below 1e-3,
+which are counted and printed.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from parity_util import compare_accept, sub_workload
+from workloads import generate, get_config
+
+pytestmark = pytest.mark.gpu
+
+TOL_LOGIT, TOL_PROB, TOL_ATTN_BF16, TOL_ATTN_F32, TOL_LSE = 2e-2, 1e-4, 2e-2, 5e-3, 1e-3
+REPORT = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out", "parity_report.jsonl")
+
+
+def _report(entry):
+    try:
+        os.makedirs(os.path.dirname(REPORT), exist_ok=True)
+        with open(REPORT, "a") as f:
+            f.write(json.dumps(entry) + "\n")
+    except OSError:
+        pass
+    print(entry)
+
+
+def run_case(name, subset=None, check_determinism=True):
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = get_config(name)
+    w = generate(cfg, device="cuda")
+    pools_before = (w["k_pages"].clone(), w["v_pages"].clone())
+    seq_before = w["seq_lens"].clone()
+    step = VerifyStep.for_workload(cfg, w, want_logits=True, want_probs=True, want_attn_f32=True)
+    step.run(w, commit=True)
+    torch.cuda.synchronize()
+    assert int(step.dev_status.item()) == 0
+
+    idx = list(range(cfg.batch)) if subset is None else subset
+    # the oracle sees the inputs as they were before the step
+    w_ref = dict(w)
+    w_ref["k_pages"], w_ref["v_pages"] = pools_before
+    w_ref["seq_lens"] = seq_before
+    ref = oracle.verify_step(sub_workload(w_ref, idx), cfg.temperature)
+    R, V = cfg.rows, cfg.vocab
+    sel = torch.as_tensor(idx, device="cuda")
+
+    entry = dict(config=name, sequences=len(idx))
+    # -- appended cache bytes: every position < L + R of the checked sequences, bit-exact
+    kp, vp = oracle.bf16_bits(w["k_pages"]), oracle.bf16_bits(w["v_pages"])
+    pt = w["page_table"].cpu().numpy()
+    for i, b in enumerate(idx):
+        n = int(seq_before[b]) + R
+        pages = pt[b, :(n + 15) // 16]
+        assert np.array_equal(kp[pages], ref["k_pages"][pages]) and np.array_equal(vp[pages], ref["v_pages"][pages])
+    # pages of other sequences and unmapped pages are untouched unless they hold block slots
+    if subset is None:
+        assert np.array_equal(kp, ref["k_pages"]) and np.array_equal(vp, ref["v_pages"])
+    # -- attention
+    o32 = step.attn_out_f32.index_select(0, sel).cpu().double().numpy()
+    o16 = step.attn_out.index_select(0, sel).cpu().double().numpy()
+    lse = step.lse.index_select(0, sel).cpu().double().numpy()
+    entry["attn_err_f32"] = float(np.abs(o32 - ref["attn_out"]).max())
+    entry["attn_err_bf16"] = float(np.abs(o16 - ref["attn_out"]).max())
+    entry["lse_err"] = float(np.abs(lse - ref["lse"]).max())
+    # -- logits / probabilities
+    z = step.logits.index_select(0, sel).cpu().double().numpy().reshape(-1, V)
+    entry["logit_err"] = float(np.abs(z - ref["logits"]).max())
+    if cfg.temperature > 0:
+        p = step.probs.index_select(0, sel).cpu().double().numpy().reshape(-1, V)
+        entry["prob_err"] = float(np.abs(p - ref["probs"]).max())
+    # -- tokens, lengths, commit
+    toks = step.out_tokens.index_select(0, sel).cpu().numpy()
+    lens = step.accept_len.index_select(0, sel).cpu().numpy()
+    st = compare_accept(ref, toks, lens, cfg.gamma)
+    entry.update({k: v for k, v in st.items() if k != "details"})
+    entry["mean_accept_len"] = float(step.accept_len.float().mean())
+    after = w["seq_lens"].cpu().numpy()
+    assert np.array_equal(after, seq_before.cpu().numpy() + step.accept_len.cpu().numpy())
+    same = lens == ref["accept_len"]
+    assert np.array_equal(after[idx][same], ref["seq_lens_after"][same])
+    assert np.all((lens >= 1) & (lens <= R))
+
+    if check_determinism:      # a second run on the same inputs is bit-identical
+        first = (step.out_tokens.clone(), step.accept_len.clone(), step.attn_out.clone(), step.logits.clone())
+        w["seq_lens"].copy_(seq_before)
+        step.run(w, commit=False)
+        torch.cuda.synchronize()
+        assert torch.equal(first[0], step.out_tokens) and torch.equal(first[1], step.accept_len)
+        assert torch.equal(first[2], step.attn_out) and torch.equal(first[3], step.logits)
+    _report(entry)
+    assert st["hard"] == 0, st["details"]
+    assert entry["attn_err_f32"] < TOL_ATTN_F32 and entry["attn_err_bf16"] < TOL_ATTN_BF16 and entry["lse_err"] < TOL_LSE
+    assert entry["logit_err"] < TOL_LOGIT
+    if cfg.temperature > 0:
+        assert entry["prob_err"] < TOL_PROB
+    return entry
+
+
+@pytest.mark.parametrize("name", ["tiny_t0", "tiny_t1", "tiny_ragged_t0", "tiny_ragged_t1", "tiny_peaked_t1"])
+def test_tiny_configs_full_parity(name):
+    run_case(name)
+
+
+@pytest.mark.parametrize("name", ["qwen7b_b1_t0", "qwen7b_b1_t0_calibrated"])
+def test_qwen_batch1_greedy_full_parity(name):
+    e = run_case(name)
+    if name.endswith("calibrated"):
+        assert e["mean_accept_len"] >= 1.0
+
+
+@pytest.mark.parametrize("name", ["qwen7b_b16_t1", "qwen7b_b16_t1_peaked"])
+def test_qwen_batch16_sampling_full_parity(name):
+    e = run_case(name)
+    if name == "qwen7b_b16_t1":
+        # flat vocabulary: acceptance tends to 2*Phi(-1/2) = 0.617 per position -> about 2.5 tokens per pass
+        assert 1.5 < e["mean_accept_len"] < 3.6
+
+
+def test_gemma_batch32_sampled_sequences():
+    run_case("gemma12b_b32_t1", subset=[0, 7, 19, 31], check_determinism=False)
+
+
+@pytest.mark.parametrize("gamma", [3, 5, 7])
+@pytest.mark.parametrize("t", [0, 1])
+def test_long_context_sweep_sampled_sequences(gamma, t):
+    run_case(f"qwen7b_long_g{gamma}_t{t}", subset=[0, 33, 63], check_determinism=False)
+
+
+def test_rollback_then_redraft_matches_a_fresh_step():
+    """Rolling back leaves the lengths untouched, and verifying a different
+    block afterwards gives what a cache that never saw the first block gives."""
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = get_config("tiny_ragged_t1")
+    w = generate(cfg, device="cuda")
+    fresh = {k: v.clone() for k, v in w.items()}
+    step = VerifyStep.for_workload(cfg, w, want_logits=True)
+    seq0 = w["seq_lens"].clone()
+    junk = dict(w)
+    junk["k_new"] = torch.randn_like(w["k_new"].float()).to(torch.bfloat16)
+    junk["v_new"] = torch.randn_like(w["v_new"].float()).to(torch.bfloat16)
+    step.attn(junk); step.accept(junk); step.commit(w["seq_lens"], rollback=True)
+    torch.cuda.synchronize()
+    assert torch.equal(w["seq_lens"], seq0)
+    step.run(w, commit=True)
+    a = (step.attn_out.clone(), step.out_tokens.clone(), step.accept_len.clone(), w["seq_lens"].clone())
+    step2 = VerifyStep.for_workload(cfg, fresh, want_logits=True)
+    step2.run(fresh, commit=True)
+    torch.cuda.synchronize()
+    assert torch.equal(a[0], step2.attn_out) and torch.equal(a[1], step2.out_tokens)
+    assert torch.equal(a[2], step2.accept_len) and torch.equal(a[3], fresh["seq_lens"])
+
+
+def test_device_side_errors_are_reported_not_fatal():
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = get_config("tiny_t0")
+    w = generate(cfg, device="cuda")
+    step = VerifyStep.for_workload(cfg, w)
+    w["seq_lens"].fill_(w["page_table"].shape[1] * 16)          # no room for the block
+    step.attn(w)
+    torch.cuda.synchronize()
+    assert int(step.dev_status.item()) == -3
+    step.dev_status.zero_()
+    bad = torch.full_like(step.accept_len, 99)
+    from paper_2505_10526_b200 import massv_kv_commit
+    before = w["seq_lens"].clone()
+    massv_kv_commit(cfg.batch, cfg.gamma, bad, w["seq_lens"], step.dev_status)
+    torch.cuda.synchronize()
+    assert int(step.dev_status.item()) == -1 and torch.equal(before, w["seq_lens"])
+
+
+def test_gamma_zero_is_plain_decoding():
+    """With no drafts the step is one ordinary decoding step: one row, one token."""
+    from dataclasses import replace
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = replace(get_config("tiny_ragged_t0"), gamma=0, name="g0")
+    w = generate(cfg, device="cuda")
+    step = VerifyStep.for_workload(cfg, w, want_logits=True)
+    ref = oracle.verify_step({k: v.clone() for k, v in w.items()}, 0.0)
+    step.run(w)
+    torch.cuda.synchronize()
+    st = compare_accept(ref, step.out_tokens.cpu().numpy(), step.accept_len.cpu().numpy(), 0)
+    assert st["hard"] == 0 and np.all(step.accept_len.cpu().numpy() == 1)
