@@ -91,7 +91,8 @@ AcceptLayout accept_layout(const massv_accept_desc& d) {
     l.off_state = off; off += align_up((size_t)d.batch * sizeof(SeqState), kAlign);
     l.off_chunks = off; off += align_up((size_t)d.batch * l.n_chunks * sizeof(double), kAlign);
     l.off_counters = off; off += align_up((size_t)d.batch * sizeof(unsigned int), kAlign);
-    l.off_logits = off; off += align_up(M * (size_t)d.vocab * sizeof(float), kAlign);
+    l.off_logits = off;
+    if (d.temperature > 0.f) off += align_up(M * (size_t)d.vocab * sizeof(float), kAlign);
     l.total = off;
     return l;
 }
@@ -169,17 +170,19 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
     g.inv_T_log2e = sampling ? 1.4426950408889634f / desc->temperature : 0.f;
     g.hidden = static_cast<const __nv_bfloat16*>(hidden);
     g.lm_head = static_cast<const __nv_bfloat16*>(lm_head);
-    g.logits = logits_out ? logits_out : reinterpret_cast<float*>(ws + l.off_logits);
+    // fp32 logits are materialised only when the sampling pass or the caller needs them
+    g.logits = logits_out ? logits_out : (sampling ? reinterpret_cast<float*>(ws + l.off_logits) : nullptr);
     g.n_part = l.n_part;
     g.part_max = reinterpret_cast<float*>(ws + l.off_max);
     g.part_sum = reinterpret_cast<float*>(ws + l.off_sum);
     g.part_idx = reinterpret_cast<int32_t*>(ws + l.off_idx);
     g.dev_status = dev_status;
-    if (launch_lm_head(g, s) != cudaSuccess) return MASSV_ERR_CUDA;
+    int n_part_used = 0;
+    if (launch_lm_head(g, s, &n_part_used) != cudaSuccess) return MASSV_ERR_CUDA;
 
     AcceptParams a;
     a.B = desc->batch; a.gamma = desc->gamma; a.V = desc->vocab; a.T = desc->temperature;
-    a.n_part = l.n_part; a.part_max = g.part_max; a.part_sum = g.part_sum; a.part_idx = g.part_idx;
+    a.n_part = n_part_used; a.part_max = g.part_max; a.part_sum = g.part_sum; a.part_idx = g.part_idx;
     a.logits = g.logits;
     a.draft_tokens = draft_tokens; a.draft_probs = draft_probs; a.u_accept = u_accept; a.u_sample = u_sample;
     a.out_tokens = out_tokens; a.accept_len = accept_len; a.probs_out = probs_out;

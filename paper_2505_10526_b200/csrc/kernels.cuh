@@ -36,8 +36,9 @@ struct LmHeadParams {
     int32_t* part_idx;              // [n_part, M]
     int32_t* dev_status;
 };
-int lm_head_num_partials(int M, int V);            // slots the kernel fills for this shape
-cudaError_t launch_lm_head(const LmHeadParams& p, cudaStream_t stream);
+int lm_head_num_partials(int M, int V);            // upper bound of the partial slots, for workspace sizing
+// *n_part_used receives the number of slots this launch fills (<= p.n_part).
+cudaError_t launch_lm_head(const LmHeadParams& p, cudaStream_t stream, int* n_part_used);
 
 // ---------------------------------------------------------------- acceptance
 struct AcceptParams {

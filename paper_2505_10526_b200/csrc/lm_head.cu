@@ -1,92 +1,506 @@
-// LM head, first correct version: z[m,v] = sum_k hidden[m,k] * lm_head[v,k] on
-// CUDA cores with fp32 accumulation, followed by per-tile softmax statistics
-// (max, sum of exponentials, argmax) over 128-entry vocabulary tiles.
-// (Sec. 2.1: the target computes p(. | X_{1:t+i-1}) for i = 1..gamma+1.)
+// LM head on the 5th-generation tensor cores with the softmax statistics fused
+// into the epilogue (Sec. 2.1: the target computes p(. | X_{1:t+i-1}) over the
+// vocabulary for the gamma+1 block rows).
+//
+//   z[m, v] = sum_k hidden[m, k] * lm_head[v, k]        bf16 x bf16 -> fp32
+//
+// Operands are swapped so that the vocabulary runs along the MMA M axis: one
+// tcgen05.mma computes D[128 vocab rows, N token rows] with the accumulator in
+// tensor memory (lane = vocab row, column = token row).  The weight matrix is
+// streamed exactly once: each persistent CTA owns a contiguous band of vocab
+// rows, cut into 128-row tiles (plus one shorter tail tile so that all bands
+// are equally long), and walks K in 64-element blocks through a TMA -> shared
+// memory ring.  Warp roles: warp 0 issues TMA loads, warp 1 issues MMAs and owns
+// the TMEM allocation, warps 2-5 drain finished accumulators (double buffered)
+// with tcgen05.ld, store fp32 logits when they are needed, and keep running
+// (max, sum exp((z-max)/T), argmax) per token row in shared memory.  At the end
+// each epilogue warp writes its statistics to its own partial slot; the
+// acceptance kernel merges the slots.  Every reduction has a fixed order.
+#include <cuda.h>
+
 #include "kernels.cuh"
 
 namespace massv {
 
 namespace {
 
-constexpr int kRowsPerIter = 8;
+constexpr int kThreads = 192;
+constexpr int kBlockK = 64;                 // bf16 elements per 128-byte swizzled row
+constexpr int kTileBytesW = kVocabTile * kBlockK * 2;
+constexpr int kMaxStages = 12;
+constexpr int kMaxCtas = 192;               // partial slots are sized for at most this many CTAs
+constexpr int kRingBytes = 200 * 1024;      // shared memory given to the TMA ring
+constexpr uint32_t kSpinLimit = 1u << 24;
 
-// One warp per vocabulary row, 8 token rows at a time.
-__global__ void __launch_bounds__(256) lm_head_naive_kernel(LmHeadParams p) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int v = blockIdx.x * 8 + warp;
-    if (v >= p.V) return;
-    const uint4* w = reinterpret_cast<const uint4*>(p.lm_head + (size_t)v * p.K);
-    const int chunks = p.K / 8;   // 16-byte words per row
-    for (int m0 = 0; m0 < p.M; m0 += kRowsPerIter) {
-        float acc[kRowsPerIter];
-        for (int r = 0; r < kRowsPerIter; ++r) acc[r] = 0.f;
-        for (int c = lane; c < chunks; c += 32) {
-            const uint4 wv = __ldg(w + c);
-            const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
-            float wf[8];
-            for (int e = 0; e < 4; ++e) { const float2 f = __bfloat1622float2(wp[e]); wf[2 * e] = f.x; wf[2 * e + 1] = f.y; }
-            for (int r = 0; r < kRowsPerIter; ++r) {
-                if (m0 + r >= p.M) break;
-                const uint4 hv = __ldg(reinterpret_cast<const uint4*>(p.hidden + (size_t)(m0 + r) * p.K) + c);
-                const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
-                for (int e = 0; e < 4; ++e) {
-                    const float2 f = __bfloat1622float2(hp[e]);
-                    acc[r] += wf[2 * e] * f.x + wf[2 * e + 1] * f.y;
+struct UmmaParams {
+    int M, K, V;
+    int n_tile;          // token rows per MMA (multiple of 16, <= 256)
+    int n_token_tiles;   // 1 or 2
+    int n_groups;        // vocab bands
+    int rows_per_group;  // multiple of 8
+    int stages;
+    int tmem_cols;       // power of two >= 2 * n_tile
+    int greedy;
+    float scale_log2;    // log2(e) / T
+    float* logits;       // [M, V] or nullptr
+    float *part_max, *part_sum;
+    int32_t* part_idx;
+    int32_t* dev_status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls (or when another role already
+// gave up), raising the CTA's abort flag instead of spinning forever.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte
+// swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);   // start address
+    d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                         // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                         // 128-byte swizzle
+    return d;
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, one CTA.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive on an mbarrier once every MMA issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+template <int C>
+__device__ __forceinline__ void tmem_load(uint32_t taddr, uint32_t (&r)[C]);
+template <>
+__device__ __forceinline__ void tmem_load<32>(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+template <>
+__device__ __forceinline__ void tmem_load<16>(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+// Wait for outstanding tcgen05.ld; the registers are passed through so that no
+// use of them can be scheduled ahead of the wait.
+template <int C>
+__device__ __forceinline__ void tmem_wait_ld(uint32_t (&r)[C]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < C; ++j) asm volatile("" : "+r"(r[j]));
+}
+
+// ------------------------------------------------------------------ statistics
+struct Stat {
+    float m;   // max logit
+    float s;   // sum of 2^((z - m) * scale_log2)
+    int idx;   // lowest vocabulary index attaining m
+};
+
+__device__ __forceinline__ Stat stat_combine(const Stat& a, const Stat& b, float scale_log2, bool greedy) {
+    Stat r;
+    const bool a_wins = a.m > b.m || (a.m == b.m && a.idx < b.idx);
+    r.m = a_wins ? a.m : b.m;
+    r.idx = a_wins ? a.idx : b.idx;
+    r.s = 0.f;
+    if (!greedy) {
+        // the loser's mass is rescaled to the winner's reference; -inf entries carry s == 0
+        const float lo = a_wins ? b.m : a.m;
+        const float s_hi = a_wins ? a.s : b.s, s_lo = a_wins ? b.s : a.s;
+        const float f = (lo == -INFINITY) ? 0.f : exp2f((lo - r.m) * scale_log2);
+        r.s = s_hi + s_lo * f;
+    }
+    return r;
+}
+
+__device__ __forceinline__ Stat stat_shfl_xor(const Stat& a, int offset, bool greedy) {
+    Stat r;
+    r.m = __shfl_xor_sync(0xffffffffu, a.m, offset);
+    r.idx = __shfl_xor_sync(0xffffffffu, a.idx, offset);
+    r.s = greedy ? 0.f : __shfl_xor_sync(0xffffffffu, a.s, offset);
+    return r;
+}
+
+// Reduce C columns (one value per lane = vocab row) across the 32 lanes of the
+// warp.  Each step halves the number of columns a lane keeps by trading the
+// other half with its partner, so the whole reduction costs about one exchange
+// per column.  On return lane l holds the warp's statistic of column l (C == 32)
+// or l >> 1 (C == 16) in v[0].
+template <int C>
+__device__ __forceinline__ void transposed_reduce(Stat (&v)[C], int lane, float scale_log2, bool greedy) {
+    int n = C;
+#pragma unroll
+    for (int offset = 16; offset >= 1; offset >>= 1) {
+        if (n > 1) {
+            const int half = n / 2;
+            const bool upper = (lane & offset) != 0;
+#pragma unroll
+            for (int i = 0; i < C / 2; ++i) {
+                if (i < half) {
+                    const Stat send = upper ? v[i] : v[i + half];
+                    const Stat keep = upper ? v[i + half] : v[i];
+                    const Stat recv = stat_shfl_xor(send, offset, greedy);
+                    v[i] = stat_combine(keep, recv, scale_log2, greedy);
                 }
             }
-        }
-        for (int r = 0; r < kRowsPerIter; ++r) {
-            float s = acc[r];
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (lane == 0 && m0 + r < p.M) p.logits[(size_t)(m0 + r) * p.V + v] = s;
+            n = half;
+        } else {
+            const Stat recv = stat_shfl_xor(v[0], offset, greedy);
+            v[0] = stat_combine(v[0], recv, scale_log2, greedy);
         }
     }
 }
 
-// grid (n_tiles, M): statistics of one 128-entry tile of one row.
-__global__ void __launch_bounds__(kVocabTile) tile_stats_kernel(LmHeadParams p) {
-    const int tile = blockIdx.x, m = blockIdx.y, t = threadIdx.x;
-    const int v = tile * kVocabTile + t;
-    __shared__ float s_val[kVocabTile];
-    __shared__ int s_idx[kVocabTile];
-    const float z = v < p.V ? p.logits[(size_t)m * p.V + v] : -INFINITY;
-    s_val[t] = z;
-    s_idx[t] = v;
-    __syncthreads();
-    for (int w = kVocabTile / 2; w > 0; w >>= 1) {
-        if (t < w) {
-            const float a = s_val[t], b = s_val[t + w];
-            if (b > a || (b == a && s_idx[t + w] < s_idx[t])) { s_val[t] = b; s_idx[t] = s_idx[t + w]; }
+struct TileCtx {
+    int v0;        // first vocabulary row of the tile
+    int rows;      // valid rows (multiple of 8, <= 128)
+};
+
+// Drain one chunk of C accumulator columns of the current tile.
+template <int C>
+__device__ __forceinline__ void drain_chunk(const UmmaParams& p, uint32_t taddr, int lane, int row_in_tile,
+                                            const TileCtx& tile, int tok0, Stat& running) {
+    uint32_t r[C];
+    tmem_load<C>(taddr, r);
+    tmem_wait_ld<C>(r);
+    const int vrow = tile.v0 + row_in_tile;
+    const bool row_ok = row_in_tile < tile.rows;
+    if (p.logits != nullptr && row_ok) {
+#pragma unroll
+        for (int j = 0; j < C; ++j) {
+            const int tok = tok0 + j;
+            if (tok < p.M) p.logits[(size_t)tok * p.V + vrow] = __uint_as_float(r[j]);
         }
-        __syncthreads();
     }
-    const float mx = s_val[0];
-    const int amax = s_idx[0];
+    Stat v[C];
+#pragma unroll
+    for (int j = 0; j < C; ++j) {
+        v[j].m = row_ok ? __uint_as_float(r[j]) : -INFINITY;
+        v[j].s = row_ok ? 1.f : 0.f;
+        v[j].idx = row_ok ? vrow : 0x7fffffff;
+    }
+    const bool greedy = p.greedy != 0;
+    transposed_reduce<C>(v, lane, p.scale_log2, greedy);
+    running = stat_combine(running, v[0], p.scale_log2, greedy);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_constant__ CUtensorMap map_w8,
+                    const __grid_constant__ CUtensorMap map_h, const UmmaParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t tmem_full_bar[2];
+    __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ float run_m[4][256];
+    __shared__ float run_s[4][256];
+    __shared__ int run_i[4][256];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int stage_bytes = kTileBytesW + p.n_tile * 128;
+    const int num_kb = p.K / kBlockK;
+
+    // which band of vocabulary rows and which token tile this CTA owns
+    const int group = blockIdx.x / p.n_token_tiles;
+    const int token_tile = blockIdx.x % p.n_token_tiles;
+    const int row_begin = min(p.V, group * p.rows_per_group);
+    const int row_end = min(p.V, row_begin + p.rows_per_group);
+    const int n_tiles = (row_end - row_begin + kVocabTile - 1) / kVocabTile;
+    const int tok_base = token_tile * p.n_tile;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
     __syncthreads();
-    float e = 0.f;
-    if (!p.greedy && v < p.V) e = exp2f((z - mx) * p.inv_T_log2e);
-    s_val[t] = e;
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abort_ptr = &abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint64_t pol_stream, pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int v0 = row_begin + t * kVocabTile;
+                const int rows = min(kVocabTile, row_end - v0);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (it / p.stages) & 1u;
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_ptr)) { ok = false; break; }
+                    uint8_t* w_dst = smem + (size_t)s * stage_bytes;
+                    uint8_t* h_dst = w_dst + kTileBytesW;
+                    mbar_expect_tx(&full_bar[s], (uint32_t)(rows * 128 + p.n_tile * 128));
+                    if (rows == kVocabTile) {
+                        tma_load_2d(w_dst, &map_w128, kb * kBlockK, v0, &full_bar[s], pol_stream);
+                    } else {
+                        for (int r = 0; r < rows; r += 8)
+                            tma_load_2d(w_dst + r * 128, &map_w8, kb * kBlockK, v0 + r, &full_bar[s], pol_stream);
+                    }
+                    tma_load_2d(h_dst, &map_h, kb * kBlockK, tok_base, &full_bar[s], pol_keep);
+                }
+            }
+            if (!ok) {
+                // let copies that are still in flight land before the CTA retires
+                for (int i = 0; i < 64; ++i) __nanosleep(2000);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) |
+                                   ((uint32_t)(kVocabTile >> 4) << 24);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int buf = t & 1;
+                if (!mbar_wait(&tmem_empty_bar[buf], (((uint32_t)t >> 1) & 1u) ^ 1u, abort_ptr)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.n_tile);
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const int s = it % p.stages;
+                    const uint32_t ph = (it / p.stages) & 1u;
+                    if (!mbar_wait(&full_bar[s], ph, abort_ptr)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint32_t b_addr = a_addr + kTileBytesW;
+#pragma unroll
+                    for (int k = 0; k < kBlockK / 16; ++k) {
+                        umma_bf16(d_tmem, umma_desc_k_sw128(a_addr + k * 32), umma_desc_k_sw128(b_addr + k * 32), idesc,
+                                  (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
+                }
+                if (ok) umma_commit(&tmem_full_bar[buf]);
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                 // TMEM lanes this warp may touch: 32*quarter ..
+        const int row_in_tile = quarter * 32 + lane;
+        const int n_chunks32 = p.n_tile / 32;
+        const bool tail16 = (p.n_tile % 32) != 0;
+        const bool greedy = p.greedy != 0;
+        // running statistics of this warp: entry [c] belongs to the lane that holds column c after a reduce
+        for (int c = lane; c < 256; c += 32) { run_m[quarter][c] = -INFINITY; run_s[quarter][c] = 0.f; run_i[quarter][c] = 0x7fffffff; }
+        __syncwarp();
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int buf = t & 1;
+            if (!mbar_wait(&tmem_full_bar[buf], ((uint32_t)t >> 1) & 1u, abort_ptr)) { ok = false; break; }
+            tc_fence_after();
+            TileCtx tile;
+            tile.v0 = row_begin + t * kVocabTile;
+            tile.rows = min(kVocabTile, row_end - tile.v0);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.n_tile);
+            for (int c = 0; c < n_chunks32; ++c) {
+                const int col = c * 32 + lane;
+                Stat running{run_m[quarter][col], run_s[quarter][col], run_i[quarter][col]};
+                drain_chunk<32>(p, taddr + c * 32, lane, row_in_tile, tile, tok_base + c * 32, running);
+                run_m[quarter][col] = running.m; run_s[quarter][col] = running.s; run_i[quarter][col] = running.idx;
+            }
+            if (tail16) {
+                // lanes 2c and 2c+1 both end up with column c of the 16-column tail; the even lane keeps it
+                const int col = n_chunks32 * 32 + (lane >> 1);
+                Stat running{run_m[quarter][col], run_s[quarter][col], run_i[quarter][col]};
+                drain_chunk<16>(p, taddr + n_chunks32 * 32, lane, row_in_tile, tile, tok_base + n_chunks32 * 32, running);
+                __syncwarp();
+                if ((lane & 1) == 0) { run_m[quarter][col] = running.m; run_s[quarter][col] = running.s; run_i[quarter][col] = running.idx; }
+                __syncwarp();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty_bar[buf]);
+        }
+        // this warp's statistics go to partial slot (group, quarter)
+        __syncwarp();
+        const size_t slot = (size_t)(group * 4 + quarter) * p.M;
+        for (int c = lane; c < p.n_tile; c += 32) {
+            const int tok = tok_base + c;
+            if (tok < p.M) {
+                p.part_max[slot + tok] = run_m[quarter][c];
+                p.part_sum[slot + tok] = greedy ? 0.f : run_s[quarter][c];
+                p.part_idx[slot + tok] = run_i[quarter][c];
+            }
+        }
+    }
+
+    tc_fence_before();
     __syncthreads();
-    for (int w = kVocabTile / 2; w > 0; w >>= 1) {
-        if (t < w) s_val[t] += s_val[t + w];
-        __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
     }
-    if (t == 0) {
-        p.part_max[(size_t)tile * p.M + m] = mx;
-        p.part_sum[(size_t)tile * p.M + m] = s_val[0];
-        p.part_idx[(size_t)tile * p.M + m] = amax;
-    }
+    if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    return fn;
+}
+
+// 2-D bf16 tensor [rows, cols] (cols contiguous), box [box_rows, 64 cols], 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (n) return n;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        n = 148;
+    return n;
 }
 
 }  // namespace
 
-int lm_head_num_partials(int M, int V) { (void)M; return (V + kVocabTile - 1) / kVocabTile; }
+// Upper bound of the partial slots the acceptance kernel may have to merge:
+// four epilogue warps per vocabulary band.
+int lm_head_num_partials(int M, int V) {
+    (void)M;
+    const int bands = (V + kVocabTile - 1) / kVocabTile;
+    return 4 * (bands < kMaxCtas ? bands : kMaxCtas);
+}
 
-cudaError_t launch_lm_head(const LmHeadParams& p, cudaStream_t stream) {
-    if (p.logits == nullptr) return cudaErrorInvalidValue;
-    lm_head_naive_kernel<<<(p.V + 7) / 8, 256, 0, stream>>>(p);
-    tile_stats_kernel<<<dim3(lm_head_num_partials(p.M, p.V), p.M), kVocabTile, 0, stream>>>(p);
-    count_launches(2);
+cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_part_used) {
+    UmmaParams p;
+    p.M = q.M; p.K = q.K; p.V = q.V;
+    p.n_token_tiles = q.M > 256 ? 2 : 1;
+    const int per_tile = (q.M + p.n_token_tiles - 1) / p.n_token_tiles;
+    p.n_tile = (per_tile + 15) / 16 * 16;
+    int ctas = sm_count();
+    if (ctas > kMaxCtas) ctas = kMaxCtas;
+    int groups = ctas / p.n_token_tiles;
+    const int bands = (q.V + kVocabTile - 1) / kVocabTile;
+    if (groups > bands) groups = bands;
+    p.n_groups = groups;
+    p.rows_per_group = ((q.V + groups - 1) / groups + 7) / 8 * 8;
+    const int stage_bytes = kTileBytesW + p.n_tile * 128;
+    int stages = kRingBytes / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    p.stages = stages;
+    int cols = 32;
+    while (cols < 2 * p.n_tile) cols *= 2;
+    p.tmem_cols = cols;
+    p.greedy = q.greedy;
+    p.scale_log2 = q.inv_T_log2e;
+    p.logits = q.logits;
+    p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
+    p.dev_status = q.dev_status;
+    if (4 * groups > q.n_part) return cudaErrorInvalidValue;
+    *n_part_used = 4 * groups;
+
+    CUtensorMap map_w128, map_w8, map_h;
+    if (!make_map(&map_w128, q.lm_head, q.V, q.K, kVocabTile) || !make_map(&map_w8, q.lm_head, q.V, q.K, 8) ||
+        !make_map(&map_h, q.hidden, q.M, q.K, p.n_tile))
+        return cudaErrorInvalidValue;
+
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    cudaError_t e = cudaFuncSetAttribute(lm_head_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    lm_head_umma_kernel<<<groups * p.n_token_tiles, kThreads, smem, stream>>>(map_w128, map_w8, map_h, p);
+    count_launches(1);
     return cudaGetLastError();
 }
 
