@@ -161,6 +161,44 @@ int massv_accept(const massv_accept_desc *desc, const void *hidden, const void *
                  void *workspace, size_t workspace_bytes, int32_t *dev_status, massv_stream_t stream);
 
 /*
+ * massv_accept for callers that have no device memory to offer as workspace and
+ * may not allocate any.  (The paper has no counterpart for this call; it exists
+ * for deployment reasons only.)
+ *
+ * Who needs it: an engine whose device pool was split up at start-up and has
+ * nothing left to lend, code that runs as a guest inside another program's CUDA
+ * context where allocating after initialisation is against the rules, and
+ * latency-critical loops that must not call cudaMalloc because it stalls the
+ * whole device.  Such callers still own the inputs and the outputs; only the
+ * scratch moves into the library.
+ *
+ * It computes exactly what massv_accept computes, with the same kernels and the
+ * same arguments, except:
+ *   - there is no workspace argument.  Scratch is a fixed array of about 640 KiB
+ *     of device memory that belongs to the library image: every GPU that loads
+ *     the library holds it until the process exits, used or not.
+ *   - the fp32 logits have no room in that array, so at T > 0 logits_out is
+ *     REQUIRED (it is an ordinary output of the caller).  At T == 0 it stays
+ *     optional.
+ *   - limits: B * (gamma + 1) <= 64, B <= 64, vocab <= 524288.  Anything larger
+ *     returns MASSV_ERR_WORKSPACE and launches nothing.
+ *   - the first call on each device looks up the array's device address (the
+ *     device that is current at the call).  Make that first call during start-up,
+ *     outside any stream capture.  Later calls on that device reuse the address.
+ *   - all calls on one device share the one array, and it keeps what the last
+ *     call left in it.  The call clears the part that has to start at zero.  Two
+ *     calls that can run on the GPU at the same time (different streams without
+ *     an ordering between them) would overwrite each other's scratch: keep calls
+ *     on one stream or order them yourself.
+ * It never calls cudaMalloc, cudaFree or any allocating routine.
+ */
+int massv_accept_static(const massv_accept_desc *desc, const void *hidden, const void *lm_head,
+                        const int32_t *draft_tokens, const float *draft_probs,
+                        const float *u_accept, const float *u_sample,
+                        int32_t *out_tokens, int32_t *accept_len, float *logits_out, float *probs_out,
+                        int32_t *dev_status, massv_stream_t stream);
+
+/*
  * Commit or roll back the speculative block (Sec. 2.1: accepted tokens are
  * added to the output and the next iteration starts from them).
  * accept_len != NULL: seq_lens[b] += accept_len[b]; cache rows of block

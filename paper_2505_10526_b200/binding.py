@@ -51,6 +51,9 @@ def _load():
     lib.massv_accept.restype = ctypes.c_int
     lib.massv_accept.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, i32p, f32p, f32p, f32p, i32p, i32p, f32p, f32p,
                                  vp, ctypes.c_size_t, i32p, vp]
+    lib.massv_accept_static.restype = ctypes.c_int
+    lib.massv_accept_static.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, i32p, f32p, f32p, f32p, i32p, i32p, f32p, f32p,
+                                        i32p, vp]
     lib.massv_kv_commit.restype = ctypes.c_int
     lib.massv_kv_commit.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, vp]
     lib.massv_strerror.restype = ctypes.c_char_p
@@ -140,6 +143,20 @@ def massv_accept(desc, hidden, lm_head, draft_tokens, draft_probs, u_accept, u_s
                            _ptr(dev_status, i32), _stream())
     if rc != 0:
         raise MassvError(rc, "massv_accept")
+
+
+def massv_accept_static(desc, hidden, lm_head, draft_tokens, draft_probs, u_accept, u_sample, out_tokens, accept_len,
+                        logits_out=None, probs_out=None, dev_status=None) -> None:
+    """massv_accept without a workspace: scratch is a fixed array inside the
+    library (for callers that cannot allocate device memory).  Needs logits_out
+    at T > 0; small problems only (see include/massv.h)."""
+    bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
+    rc = _lib.massv_accept_static(ctypes.byref(desc), _ptr(hidden, bf), _ptr(lm_head, bf), _ptr(draft_tokens, i32),
+                                  _ptr(draft_probs, f32), _ptr(u_accept, f32), _ptr(u_sample, f32),
+                                  _ptr(out_tokens, i32), _ptr(accept_len, i32), _ptr(logits_out, f32),
+                                  _ptr(probs_out, f32), _ptr(dev_status, i32), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_accept_static")
 
 
 def massv_kv_commit(batch, gamma, accept_len, seq_lens, dev_status=None) -> None:
