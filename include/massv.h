@@ -67,7 +67,7 @@ typedef struct massv_attn_desc {
     int32_t max_pages_per_seq;   /* row length of page_table */
     int64_t num_pages;           /* pages in the pool */
     float scale;                 /* score scale; 0 selects 1/sqrt(d) */
-    int32_t kv_chunk;            /* tokens per split of the KV scan, multiple of 64; 0 = choose automatically */
+    int32_t kv_chunk;            /* tokens per split of the KV scan, multiple of 64, <= 4096; 0 = choose automatically */
     uint32_t flags;              /* reserved, 0 */
 } massv_attn_desc;
 

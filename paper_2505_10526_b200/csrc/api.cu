@@ -40,7 +40,7 @@ int check_attn_desc(const massv_attn_desc* d) {
     if (d->head_dim != 64 && d->head_dim != 128 && d->head_dim != 256) return MASSV_ERR_UNSUPPORTED;
     if (d->n_q_heads % d->n_kv_heads != 0) return MASSV_ERR_UNSUPPORTED;
     if ((d->n_q_heads / d->n_kv_heads) * (d->gamma + 1) > 64) return MASSV_ERR_UNSUPPORTED;
-    if (d->kv_chunk % 64 != 0) return MASSV_ERR_UNSUPPORTED;
+    if (d->kv_chunk % 64 != 0 || d->kv_chunk > 4096) return MASSV_ERR_UNSUPPORTED;
     if (d->flags != 0) return MASSV_ERR_UNSUPPORTED;
     return MASSV_OK;
 }
