@@ -16,6 +16,7 @@ namespace massv {
 namespace {
 
 constexpr int kScanThreads = 256;
+constexpr int kScanBatch = 6;     // partial slots a lane loads before merging (192 slots = one batch)
 constexpr int kSampleThreads = 256;
 constexpr int kPerThread = kResidualChunk / kSampleThreads;   // 16 contiguous entries per thread
 static_assert(kPerThread == 16, "chunk layout");
@@ -36,55 +37,74 @@ __device__ __forceinline__ Stat combine(Stat a, Stat b, float inv_T) {
     return r;
 }
 
-// One CTA per sequence.
+// One CTA per sequence, one warp per block row.  Each lane merges a strided
+// share of the partial slots (independent loads), a butterfly merges the lanes,
+// and warp 0 then evaluates all gamma accept tests at once (lane j = draft j) and
+// takes the first failure.
 __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams p) {
-    const int b = blockIdx.x, t = threadIdx.x;
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int R = p.gamma + 1, M = p.B * R;
     const bool greedy = !(p.T > 0.f);
     const float inv_T = greedy ? 1.f : 1.f / p.T;
-    __shared__ Stat red[kScanThreads];
     __shared__ Stat row_stat[kMaxRows];
+    static_assert(kScanThreads / 32 >= kMaxRows, "one warp per block row");
 
-    for (int j = 0; j < R; ++j) {
-        const int row = b * R + j;
+    if (warp < R) {
+        const int row = b * R + warp;
         Stat acc{-INFINITY, 0.f, 0x7fffffff};
-        for (int i = t; i < p.n_part; i += kScanThreads) {
-            Stat x{p.part_max[(size_t)i * M + row], greedy ? 0.f : p.part_sum[(size_t)i * M + row],
-                   p.part_idx[(size_t)i * M + row]};
-            acc = combine(acc, x, inv_T);
+        for (int i0 = 0; i0 < p.n_part; i0 += 32 * kScanBatch) {
+            // issue a batch of independent loads before merging them
+            Stat x[kScanBatch];
+#pragma unroll
+            for (int k = 0; k < kScanBatch; ++k) {
+                const int i = i0 + k * 32 + lane;
+                x[k] = Stat{-INFINITY, 0.f, 0x7fffffff};
+                if (i < p.n_part) {
+                    x[k].m = p.part_max[(size_t)i * M + row];
+                    x[k].s = greedy ? 0.f : p.part_sum[(size_t)i * M + row];
+                    x[k].idx = p.part_idx[(size_t)i * M + row];
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < kScanBatch; ++k) acc = combine(acc, x[k], inv_T);
         }
-        red[t] = acc;
-        __syncthreads();
-        for (int w = kScanThreads / 2; w > 0; w >>= 1) {
-            if (t < w) red[t] = combine(red[t], red[t + w], inv_T);
-            __syncthreads();
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            Stat y;
+            y.m = __shfl_xor_sync(0xffffffffu, acc.m, o);
+            y.s = __shfl_xor_sync(0xffffffffu, acc.s, o);
+            y.idx = __shfl_xor_sync(0xffffffffu, acc.idx, o);
+            // both partners must form the same sum: order the operands by lane
+            acc = (lane & o) ? combine(y, acc, inv_T) : combine(acc, y, inv_T);
         }
-        if (t == 0) row_stat[j] = red[0];
-        __syncthreads();
+        if (lane == 0) row_stat[warp] = acc;
     }
-    if (t != 0) return;
+    __syncthreads();
+    if (warp != 0) return;
 
-    int n = p.gamma;
-    int32_t* toks = p.out_tokens + (size_t)b * R;
-    for (int j = 0; j < R; ++j) toks[j] = -1;
-    for (int j = 0; j < p.gamma; ++j) {
-        const int x = p.draft_tokens[(size_t)b * p.gamma + j];
-        bool ok;
+    bool ok = true;
+    int x = -1;
+    if (lane < p.gamma) {
+        x = p.draft_tokens[(size_t)b * p.gamma + lane];
         if (x < 0 || x >= p.V) {
             set_status(p.dev_status, MASSV_ERR_INVALID_ARG);
             ok = false;
         } else if (greedy) {
-            ok = (x == row_stat[j].idx);
+            ok = (x == row_stat[lane].idx);
         } else {
-            const float zx = p.logits[(size_t)(b * R + j) * p.V + x];
-            const float px = expf((zx - row_stat[j].m) * inv_T) / row_stat[j].s;
-            const float qx = p.draft_probs[((size_t)b * p.gamma + j) * p.V + x];
-            const float lhs = p.u_accept[(size_t)b * p.gamma + j] * qx;
+            const float zx = p.logits[(size_t)(b * R + lane) * p.V + x];
+            const float px = expf((zx - row_stat[lane].m) * inv_T) / row_stat[lane].s;
+            const float qx = p.draft_probs[((size_t)b * p.gamma + lane) * p.V + x];
+            const float lhs = p.u_accept[(size_t)b * p.gamma + lane] * qx;
             ok = lhs < px;
         }
-        if (!ok) { n = j; break; }
-        toks[j] = x;
     }
+    const unsigned fail = __ballot_sync(0xffffffffu, !ok);
+    const int n = fail ? (__ffs(fail) - 1) : p.gamma;       // first rejected draft, or gamma if none
+    int32_t* toks = p.out_tokens + (size_t)b * R;
+    if (lane < R) toks[lane] = lane < n ? x : -1;
+    __syncwarp();
+    if (lane != 0) return;
     p.accept_len[b] = n + 1;
     if (greedy) {
         toks[n] = row_stat[n].idx;

@@ -13,7 +13,8 @@
 // online softmax in registers: warp (mt, ts) owns 16 query rows and a 64/TS-token
 // slice of every tile.  Partial (max, sum, O) of the warps are merged through
 // shared memory; sequences that span several chunks are merged by a second
-// kernel.  All reductions have a fixed order.
+// kernel.  The block's own K/V rows are appended by the CTA whose chunk holds
+// their positions.  All reductions have a fixed order.
 #include "kernels.cuh"
 #include "ptx.cuh"
 
@@ -23,30 +24,6 @@ namespace {
 
 constexpr int kTile = 64;            // tokens per pipeline stage
 constexpr int kMaxChunkPages = 256;  // kv_chunk <= 4096 tokens
-
-__device__ __forceinline__ size_t kv_offset(const AttnParams& p, int b, int pos, int g, int32_t* bad) {
-    const int page = p.page_table[(size_t)b * p.max_pages + pos / kPageSize];
-    if (page < 0 || page >= p.num_pages) { *bad = 1; return 0; }
-    return (((size_t)page * p.Hkv + g) * kPageSize + (pos % kPageSize)) * p.d;
-}
-
-// Store the block's K/V rows at cache positions L_b .. L_b+gamma.
-__global__ void kv_append_kernel(AttnParams p) {
-    // one CTA per (sequence, row); threads copy Hkv*d elements as 16-byte words
-    const int b = blockIdx.x / p.R, j = blockIdx.x % p.R;
-    const int L = p.seq_lens[b];
-    if (L < 0 || L + p.R > p.max_pages * kPageSize) { set_status(p.dev_status, MASSV_ERR_CAPACITY); return; }
-    const int words = p.d / 8;
-    for (int i = threadIdx.x; i < p.Hkv * words; i += blockDim.x) {
-        const int g = i / words, w = i % words;
-        int32_t bad = 0;
-        const size_t dst = kv_offset(p, b, L + j, g, &bad);
-        if (bad) { set_status(p.dev_status, MASSV_ERR_CAPACITY); continue; }
-        const size_t src = (((size_t)b * p.R + j) * p.Hkv + g) * p.d;
-        reinterpret_cast<uint4*>(p.k_pages + dst)[w] = reinterpret_cast<const uint4*>(p.k_new + src)[w];
-        reinterpret_cast<uint4*>(p.v_pages + dst)[w] = reinterpret_cast<const uint4*>(p.v_new + src)[w];
-    }
-}
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -102,7 +79,10 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int L = p.seq_lens[b];
-    if (L < 0 || L + p.R > p.max_pages * kPageSize) return;      // reported by the append kernel
+    if (L < 0 || L + p.R > p.max_pages * kPageSize) {            // no room for the block: skip the sequence
+        if (chunk == 0 && g == 0 && threadIdx.x == 0) set_status(p.dev_status, MASSV_ERR_CAPACITY);
+        return;
+    }
     const int n_ctx = L + p.R;
     const int c_begin = chunk * p.kv_chunk;
     if (c_begin >= n_ctx) return;
@@ -201,11 +181,31 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
             const int valid = min(kTile, c_end - tile_start);
             uint8_t* kst = smem + (size_t)s * Cfg::kStageBytes;
             uint8_t* vst = kst + Cfg::kBytesK;
-            if (valid < kTile) {
+            if (tile_start + kTile > L) {
+                constexpr int UPR = D / 8;
+                // Append: the block's K/V rows (positions L .. L+gamma) are not in the cache yet.
+                // The warp that owns those tokens puts them into the tile in shared memory, and
+                // the mt == 0 warp also stores them to their page slots.
+                const int p_first = max(L, tile_start + ts * NT), p_last = min(n_ctx, tile_start + ts * NT + NT);
+                for (int i = lane; i < (p_last - p_first) * UPR; i += 32) {
+                    const int pos = p_first + i / UPR, u = i % UPR, row = pos - tile_start;
+                    const size_t src = (((size_t)b * p.R + (pos - L)) * p.Hkv + g) * D + u * 8;
+                    const uint4 kv = *reinterpret_cast<const uint4*>(p.k_new + src);
+                    const uint4 vv = *reinterpret_cast<const uint4*>(p.v_new + src);
+                    *reinterpret_cast<uint4*>(kst + (u / 8) * Cfg::kRegion + swz(row, u % 8)) = kv;
+                    *reinterpret_cast<uint4*>(vst + (u / 8) * Cfg::kRegion + swz(row, u % 8)) = vv;
+                    if (mt == 0) {
+                        const int pid = s_pages[(pos - c_begin) / kPageSize];
+                        if (pid >= 0 && pid < p.num_pages) {
+                            const size_t dst = (((size_t)pid * p.Hkv + g) * kPageSize + (pos % kPageSize)) * D + u * 8;
+                            *reinterpret_cast<uint4*>(p.k_pages + dst) = kv;
+                            *reinterpret_cast<uint4*>(p.v_pages + dst) = vv;
+                        }
+                    }
+                }
                 // Rows past the end of the context hold stale bytes; their weights are zero, but
                 // 0 * NaN would still poison P V, so clear the V rows this warp will read.
                 const int first = max(valid, ts * NT), last = ts * NT + NT;
-                constexpr int UPR = D / 8;
                 for (int i = lane; i < (last - first) * UPR; i += 32) {
                     const int row = first + i / UPR, u = i % UPR;
                     *reinterpret_cast<uint4*>(vst + (u / 8) * Cfg::kRegion + swz(row, u % 8)) = make_uint4(0u, 0u, 0u, 0u);
@@ -359,31 +359,44 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 
 // Merge the chunks of sequences that span more than one: one CTA per
 // (sequence, KV head, query row), one thread per channel.
-__global__ void attn_combine_kernel(const AttnParams p, int rows_pad) {
+constexpr int kCombineMaxChunks = 1024;
+__global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, int rows_pad) {
     const int G = p.Hq / p.Hkv, rows = G * p.R;
     const int r = blockIdx.x % rows, g = (blockIdx.x / rows) % p.Hkv, b = blockIdx.x / (rows * p.Hkv);
     const int L = p.seq_lens[b];
     if (L < 0 || L + p.R > p.max_pages * kPageSize) return;
     const int n_chunks = (L + p.R + p.kv_chunk - 1) / p.kv_chunk;
     if (n_chunks <= 1) return;
+    __shared__ float s_w[kCombineMaxChunks];    // first the chunk maxima, then the merge weights
+    __shared__ float s_l[kCombineMaxChunks];
     const size_t item0 = ((size_t)b * p.Hkv + g) * p.max_chunks;
+    for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) {
+        const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((item0 + c) * rows_pad + r) * 2);
+        s_w[c] = ml.x;
+        s_l[c] = ml.y;
+    }
+    __syncthreads();
     float M = -INFINITY;
-    for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, p.part_ml[((item0 + c) * rows_pad + r) * 2]);
+    for (int c = 0; c < n_chunks; ++c) M = fmaxf(M, s_w[c]);
+    __syncthreads();
+    for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) s_w[c] = s_w[c] == -INFINITY ? 0.f : exp2f(s_w[c] - M);
+    __syncthreads();
+    float Lsum = 0.f;
+    for (int c = 0; c < n_chunks; ++c) Lsum += s_l[c] * s_w[c];
+    const float inv = 1.f / Lsum;
     const int j = r / G, hh = r % G;
     const size_t row_out = ((size_t)b * p.R + j) * p.Hq + g * G + hh;
-    float Lsum = 0.f;
-    for (int c = 0; c < n_chunks; ++c) {
-        const float mc = p.part_ml[((item0 + c) * rows_pad + r) * 2];
-        Lsum += p.part_ml[((item0 + c) * rows_pad + r) * 2 + 1] * (mc == -INFINITY ? 0.f : exp2f(mc - M));
-    }
-    const float inv = 1.f / Lsum;
+    const float* src = p.part_o + (item0 * rows_pad + r) * p.d;
+    const size_t chunk_stride = (size_t)rows_pad * p.d;
     for (int col = threadIdx.x; col < p.d; col += blockDim.x) {
         float acc = 0.f;
-        for (int c = 0; c < n_chunks; ++c) {
-            const float mc = p.part_ml[((item0 + c) * rows_pad + r) * 2];
-            const float f = mc == -INFINITY ? 0.f : exp2f(mc - M);
-            acc += p.part_o[((item0 + c) * rows_pad + r) * p.d + col] * f;
+        int c = 0;
+        for (; c + 4 <= n_chunks; c += 4) {      // four independent loads in flight, summed in chunk order
+            const float v0 = src[(size_t)c * chunk_stride + col], v1 = src[(size_t)(c + 1) * chunk_stride + col];
+            const float v2 = src[(size_t)(c + 2) * chunk_stride + col], v3 = src[(size_t)(c + 3) * chunk_stride + col];
+            acc += v0 * s_w[c]; acc += v1 * s_w[c + 1]; acc += v2 * s_w[c + 2]; acc += v3 * s_w[c + 3];
         }
+        for (; c < n_chunks; ++c) acc += src[(size_t)c * chunk_stride + col] * s_w[c];
         acc *= inv;
         p.out[row_out * p.d + col] = __float2bfloat16(acc);
         if (p.out_f32) p.out_f32[row_out * p.d + col] = acc;
@@ -426,7 +439,6 @@ cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
     if (!make_tensor_map_bf16_2d(&mk, p.k_pages, rows_total, p.d, kPageSize) ||
         !make_tensor_map_bf16_2d(&mv, p.v_pages, rows_total, p.d, kPageSize))
         return cudaErrorInvalidValue;
-    kv_append_kernel<<<p.B * p.R, 128, 0, stream>>>(p);
     const int rows = (p.Hq / p.Hkv) * p.R;
     const int mt = attn_rows_pad(rows) / 16;
     cudaError_t e;
@@ -437,10 +449,11 @@ cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
         default: return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;
-    int launched = 2;
+    int launched = 1;
     if (p.max_chunks > 1) {
+        if (p.max_chunks > kCombineMaxChunks) return cudaErrorInvalidValue;
         attn_combine_kernel<<<p.B * p.Hkv * rows, p.d < 128 ? 64 : 128, 0, stream>>>(p, attn_rows_pad(rows));
-        launched = 3;
+        launched = 2;
     }
     count_launches(launched);
     return cudaGetLastError();

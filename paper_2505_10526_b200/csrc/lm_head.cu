@@ -7,15 +7,15 @@
 // Operands are swapped so that the vocabulary runs along the MMA M axis: one
 // tcgen05.mma computes D[128 vocab rows, N token rows] with the accumulator in
 // tensor memory (lane = vocab row, column = token row).  The weight matrix is
-// streamed exactly once: each persistent CTA owns a contiguous band of vocab
-// rows, cut into 128-row tiles (plus one shorter tail tile so that all bands
-// are equally long), and walks K in 64-element blocks through a TMA -> shared
-// memory ring.  Warp roles: warp 0 issues TMA loads, warp 1 issues MMAs and owns
-// the TMEM allocation, warps 2-5 drain finished accumulators (double buffered)
+// streamed exactly once: each persistent CTA owns a contiguous band of whole
+// 128-row vocabulary tiles and walks K in 64-element blocks through a TMA ->
+// shared memory ring.  Warp roles: warp 0 issues TMA loads, warp 1 issues MMAs and owns
+// the TMEM allocation, warps 2-9 drain finished accumulators (double buffered)
 // with tcgen05.ld, store fp32 logits when they are needed, and keep running
-// (max, sum exp((z-max)/T), argmax) per token row in shared memory.  At the end
-// each epilogue warp writes its statistics to its own partial slot; the
-// acceptance kernel merges the slots.  Every reduction has a fixed order.
+// (max, sum exp((z-max)/T), argmax) per token row in shared memory (warp-wide
+// integer max reduction on order-preserving keys, ballot for the argmax, a
+// transposed butterfly for the sums).  At the end the CTA writes one partial
+// slot; the acceptance kernel merges the slots.  Every reduction has a fixed order.
 #include <cuda.h>
 
 #include "kernels.cuh"
@@ -25,7 +25,8 @@ namespace massv {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kEpilogueWarps = 8;          // two per TMEM lane quarter
+constexpr int kThreads = (2 + kEpilogueWarps) * 32;
 constexpr int kBlockK = 64;                 // bf16 elements per 128-byte swizzled row
 constexpr int kTileBytesW = kVocabTile * kBlockK * 2;
 constexpr int kMaxStages = 12;
@@ -37,7 +38,7 @@ struct UmmaParams {
     int n_tile;          // token rows per MMA (multiple of 16, <= 256)
     int n_token_tiles;   // 1 or 2
     int n_groups;        // vocab bands
-    int rows_per_group;  // multiple of 8
+    int tiles_per_group; // whole 128-row tiles per band
     int stages;
     int tmem_cols;       // power of two >= 2 * n_tile
     int greedy;
@@ -133,21 +134,22 @@ __device__ __forceinline__ Stat stat_combine(const Stat& a, const Stat& b, float
     return r;
 }
 
-__device__ __forceinline__ Stat stat_shfl_xor(const Stat& a, int offset, bool greedy) {
-    Stat r;
-    r.m = __shfl_xor_sync(0xffffffffu, a.m, offset);
-    r.idx = __shfl_xor_sync(0xffffffffu, a.idx, offset);
-    r.s = greedy ? 0.f : __shfl_xor_sync(0xffffffffu, a.s, offset);
-    return r;
+// Order-preserving map float -> uint32, so that the integer warp reduction
+// (redux.sync.max.u32) yields the float maximum.
+__device__ __forceinline__ uint32_t float_key(float x) {
+    const uint32_t b = __float_as_uint(x);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// Reduce C columns (one value per lane = vocab row) across the 32 lanes of the
-// warp.  Each step halves the number of columns a lane keeps by trading the
-// other half with its partner, so the whole reduction costs about one exchange
-// per column.  On return lane l holds the warp's statistic of column l (C == 32)
-// or l >> 1 (C == 16) in v[0].
+// Sum C columns (one value per lane) across the 32 lanes of the warp.  Each step
+// halves the number of columns a lane keeps by trading the other half with its
+// partner, so the reduction costs about one exchange per column.  On return
+// lane l holds the sum of column l (C == 32) or l >> 1 (C == 16) in v[0].
 template <int C>
-__device__ __forceinline__ void transposed_reduce(Stat (&v)[C], int lane, float scale_log2, bool greedy) {
+__device__ __forceinline__ void transposed_sum(float (&v)[C], int lane) {
     int n = C;
 #pragma unroll
     for (int offset = 16; offset >= 1; offset >>= 1) {
@@ -157,16 +159,14 @@ __device__ __forceinline__ void transposed_reduce(Stat (&v)[C], int lane, float 
 #pragma unroll
             for (int i = 0; i < C / 2; ++i) {
                 if (i < half) {
-                    const Stat send = upper ? v[i] : v[i + half];
-                    const Stat keep = upper ? v[i + half] : v[i];
-                    const Stat recv = stat_shfl_xor(send, offset, greedy);
-                    v[i] = stat_combine(keep, recv, scale_log2, greedy);
+                    const float send = upper ? v[i] : v[i + half];
+                    const float keep = upper ? v[i + half] : v[i];
+                    v[i] = keep + __shfl_xor_sync(0xffffffffu, send, offset);
                 }
             }
             n = half;
         } else {
-            const Stat recv = stat_shfl_xor(v[0], offset, greedy);
-            v[0] = stat_combine(v[0], recv, scale_log2, greedy);
+            v[0] += __shfl_xor_sync(0xffffffffu, v[0], offset);
         }
     }
 }
@@ -176,7 +176,10 @@ struct TileCtx {
     int rows;      // valid rows (multiple of 8, <= 128)
 };
 
-// Drain one chunk of C accumulator columns of the current tile.
+// Drain one chunk of C accumulator columns of the current tile: store the
+// logits if asked, and fold the chunk into `running`, the statistic of the
+// column this lane owns (column `lane` of the chunk for C == 32, `lane >> 1`
+// for C == 16).
 template <int C>
 __device__ __forceinline__ void drain_chunk(const UmmaParams& p, uint32_t taddr, int lane, int row_in_tile,
                                             const TileCtx& tile, int tok0, Stat& running) {
@@ -186,27 +189,41 @@ __device__ __forceinline__ void drain_chunk(const UmmaParams& p, uint32_t taddr,
     const int vrow = tile.v0 + row_in_tile;
     const bool row_ok = row_in_tile < tile.rows;
     if (p.logits != nullptr && row_ok) {
+        float* dst = p.logits + (size_t)tok0 * p.V + vrow;
 #pragma unroll
         for (int j = 0; j < C; ++j) {
-            const int tok = tok0 + j;
-            if (tok < p.M) p.logits[(size_t)tok * p.V + vrow] = __uint_as_float(r[j]);
+            if (tok0 + j < p.M) dst[(size_t)j * p.V] = __uint_as_float(r[j]);
         }
     }
-    Stat v[C];
+    const bool greedy = p.greedy != 0;
+    const int warp_row0 = vrow - lane;          // vocabulary row of lane 0
+    float sums[C];
+    Stat mine{-INFINITY, 0.f, 0x7fffffff};
 #pragma unroll
     for (int j = 0; j < C; ++j) {
-        v[j].m = row_ok ? __uint_as_float(r[j]) : -INFINITY;
-        v[j].s = row_ok ? 1.f : 0.f;
-        v[j].idx = row_ok ? vrow : 0x7fffffff;
+        const float z = row_ok ? __uint_as_float(r[j]) + 0.f : -INFINITY;     // + 0 folds -0 into +0
+        const uint32_t key = float_key(z);
+        const uint32_t kmax = __reduce_max_sync(0xffffffffu, key);
+        const unsigned hit = __ballot_sync(0xffffffffu, key == kmax);
+        const float mx = key_float(kmax);
+        sums[j] = (greedy || mx == -INFINITY) ? 0.f : exp2f((z - mx) * p.scale_log2);
+        if ((C == 32 ? lane : (lane >> 1)) == j) {
+            mine.m = mx;
+            mine.idx = mx == -INFINITY ? 0x7fffffff : warp_row0 + (__ffs(hit) - 1);   // lowest row attaining the max
+        }
     }
-    const bool greedy = p.greedy != 0;
-    transposed_reduce<C>(v, lane, p.scale_log2, greedy);
-    running = stat_combine(running, v[0], p.scale_log2, greedy);
+    if (!greedy) {
+        transposed_sum<C>(sums, lane);
+        mine.s = sums[0];
+    }
+    running = stat_combine(running, mine, p.scale_log2, greedy);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_constant__ CUtensorMap map_w8,
-                    const __grid_constant__ CUtensorMap map_h, const UmmaParams p) {
+lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_constant__ CUtensorMap map_w64,
+                    const __grid_constant__ CUtensorMap map_w32, const __grid_constant__ CUtensorMap map_w16,
+                    const __grid_constant__ CUtensorMap map_w8, const __grid_constant__ CUtensorMap map_h,
+                    const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
@@ -226,14 +243,15 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
     // which band of vocabulary rows and which token tile this CTA owns
     const int group = blockIdx.x / p.n_token_tiles;
     const int token_tile = blockIdx.x % p.n_token_tiles;
-    const int row_begin = min(p.V, group * p.rows_per_group);
-    const int row_end = min(p.V, row_begin + p.rows_per_group);
-    const int n_tiles = (row_end - row_begin + kVocabTile - 1) / kVocabTile;
+    const int row_begin = min(p.V, group * p.tiles_per_group * kVocabTile);
+    const int row_end = min(p.V, row_begin + p.tiles_per_group * kVocabTile);
+    constexpr int tile_rows = kVocabTile;
+    const int n_tiles = (row_end - row_begin + tile_rows - 1) / tile_rows;
     const int tok_base = token_tile * p.n_tile;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], kEpilogueWarps); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -260,8 +278,8 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             uint32_t it = 0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
-                const int v0 = row_begin + t * kVocabTile;
-                const int rows = min(kVocabTile, row_end - v0);
+                const int v0 = row_begin + t * tile_rows;
+                const int rows = min(tile_rows, row_end - v0);
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const int s = it % p.stages;
                     const uint32_t ph = (it / p.stages) & 1u;
@@ -272,8 +290,12 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
                     if (rows == kVocabTile) {
                         tma_load_2d(w_dst, &map_w128, kb * kBlockK, v0, &full_bar[s], pol_stream);
                     } else {
-                        for (int r = 0; r < rows; r += 8)
-                            tma_load_2d(w_dst + r * 128, &map_w8, kb * kBlockK, v0 + r, &full_bar[s], pol_stream);
+                        // rows is a multiple of 8 below 128: one box per set bit
+                        int r = 0;
+                        if (rows & 64) { tma_load_2d(w_dst + r * 128, &map_w64, kb * kBlockK, v0 + r, &full_bar[s], pol_stream); r += 64; }
+                        if (rows & 32) { tma_load_2d(w_dst + r * 128, &map_w32, kb * kBlockK, v0 + r, &full_bar[s], pol_stream); r += 32; }
+                        if (rows & 16) { tma_load_2d(w_dst + r * 128, &map_w16, kb * kBlockK, v0 + r, &full_bar[s], pol_stream); r += 16; }
+                        if (rows & 8) { tma_load_2d(w_dst + r * 128, &map_w8, kb * kBlockK, v0 + r, &full_bar[s], pol_stream); r += 8; }
                     }
                     tma_load_2d(h_dst, &map_h, kb * kBlockK, tok_base, &full_bar[s], pol_keep);
                 }
@@ -313,31 +335,34 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             }
         }
     } else {
-        // ------------------------------------------------ epilogue (warps 2..5)
-        const int quarter = warp & 3;                 // TMEM lanes this warp may touch: 32*quarter ..
+        // ------------------------------------------------ epilogue (warps 2..9)
+        // TMEM lanes 32*quarter .. +31 are the only ones warp (quarter = warp % 4) may read; the two
+        // warps that share a quarter take alternate column chunks.
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         const int row_in_tile = quarter * 32 + lane;
         const int n_chunks32 = p.n_tile / 32;
         const bool tail16 = (p.n_tile % 32) != 0;
-        const bool greedy = p.greedy != 0;
-        // running statistics of this warp: entry [c] belongs to the lane that holds column c after a reduce
-        for (int c = lane; c < 256; c += 32) { run_m[quarter][c] = -INFINITY; run_s[quarter][c] = 0.f; run_i[quarter][c] = 0x7fffffff; }
-        __syncwarp();
+        // running statistics per (quarter, column); each column is touched by exactly one lane of one warp
+        if (half == 0)
+            for (int c = lane; c < 256; c += 32) { run_m[quarter][c] = -INFINITY; run_s[quarter][c] = 0.f; run_i[quarter][c] = 0x7fffffff; }
+        asm volatile("bar.sync 1, %0;" ::"r"(kEpilogueWarps * 32) : "memory");     // epilogue warps only
         bool ok = true;
         for (int t = 0; t < n_tiles && ok; ++t) {
             const int buf = t & 1;
             if (!mbar_wait(&tmem_full_bar[buf], ((uint32_t)t >> 1) & 1u, abort_ptr)) { ok = false; break; }
             tc_fence_after();
             TileCtx tile;
-            tile.v0 = row_begin + t * kVocabTile;
-            tile.rows = min(kVocabTile, row_end - tile.v0);
+            tile.v0 = row_begin + t * tile_rows;
+            tile.rows = min(tile_rows, row_end - tile.v0);
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.n_tile);
-            for (int c = 0; c < n_chunks32; ++c) {
+            for (int c = half; c < n_chunks32; c += 2) {
                 const int col = c * 32 + lane;
                 Stat running{run_m[quarter][col], run_s[quarter][col], run_i[quarter][col]};
                 drain_chunk<32>(p, taddr + c * 32, lane, row_in_tile, tile, tok_base + c * 32, running);
                 run_m[quarter][col] = running.m; run_s[quarter][col] = running.s; run_i[quarter][col] = running.idx;
             }
-            if (tail16) {
+            if (tail16 && (n_chunks32 & 1) == half) {
                 // lanes 2c and 2c+1 both end up with column c of the 16-column tail; the even lane keeps it
                 const int col = n_chunks32 * 32 + (lane >> 1);
                 Stat running{run_m[quarter][col], run_s[quarter][col], run_i[quarter][col]};
@@ -350,21 +375,24 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             __syncwarp();
             if (lane == 0) mbar_arrive(&tmem_empty_bar[buf]);
         }
-        // this warp's statistics go to partial slot (group, quarter)
-        __syncwarp();
-        const size_t slot = (size_t)(group * 4 + quarter) * p.M;
-        for (int c = lane; c < p.n_tile; c += 32) {
-            const int tok = tok_base + c;
-            if (tok < p.M) {
-                p.part_max[slot + tok] = run_m[quarter][c];
-                p.part_sum[slot + tok] = greedy ? 0.f : run_s[quarter][c];
-                p.part_idx[slot + tok] = run_i[quarter][c];
-            }
-        }
     }
 
     tc_fence_before();
     __syncthreads();
+    // the CTA's statistics: merge the four lane quarters (ascending rows) into one partial slot
+    for (int c = threadIdx.x; c < p.n_tile; c += kThreads) {
+        const int tok = tok_base + c;
+        if (tok < p.M) {
+            Stat acc{run_m[0][c], run_s[0][c], run_i[0][c]};
+#pragma unroll
+            for (int qd = 1; qd < 4; ++qd)
+                acc = stat_combine(acc, Stat{run_m[qd][c], run_s[qd][c], run_i[qd][c]}, p.scale_log2, p.greedy != 0);
+            const size_t slot = (size_t)group * p.M;
+            p.part_max[slot + tok] = acc.m;
+            p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
+            p.part_idx[slot + tok] = acc.idx;
+        }
+    }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
@@ -385,12 +413,11 @@ int sm_count() {
 
 }  // namespace
 
-// Upper bound of the partial slots the acceptance kernel may have to merge:
-// four epilogue warps per vocabulary band.
+// Upper bound of the partial slots the acceptance kernel may have to merge: one per CTA.
 int lm_head_num_partials(int M, int V) {
     (void)M;
     const int bands = (V + kVocabTile - 1) / kVocabTile;
-    return 4 * (bands < kMaxCtas ? bands : kMaxCtas);
+    return bands < kMaxCtas ? bands : kMaxCtas;
 }
 
 cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_part_used) {
@@ -401,11 +428,15 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.n_tile = (per_tile + 15) / 16 * 16;
     int ctas = sm_count();
     if (ctas > kMaxCtas) ctas = kMaxCtas;
+    // Whole tiles per CTA: a band with a short tail tile would run a full K loop with almost
+    // nothing in flight.  Use the fewest CTAs that still reach the minimal tiles-per-CTA count
+    // (1188 tiles on 148 SMs: 132 CTAs x 9 tiles).
     int groups = ctas / p.n_token_tiles;
     const int bands = (q.V + kVocabTile - 1) / kVocabTile;
     if (groups > bands) groups = bands;
+    p.tiles_per_group = (bands + groups - 1) / groups;
+    groups = (bands + p.tiles_per_group - 1) / p.tiles_per_group;
     p.n_groups = groups;
-    p.rows_per_group = ((q.V + groups - 1) / groups + 7) / 8 * 8;
     const int stage_bytes = kTileBytesW + p.n_tile * 128;
     int stages = kRingBytes / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
@@ -418,18 +449,18 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.logits = q.logits;
     p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
     p.dev_status = q.dev_status;
-    if (4 * groups > q.n_part) return cudaErrorInvalidValue;
-    *n_part_used = 4 * groups;
+    if (groups > q.n_part) return cudaErrorInvalidValue;
+    *n_part_used = groups;
 
-    CUtensorMap map_w128, map_w8, map_h;
-    if (!make_tensor_map_bf16_2d(&map_w128, q.lm_head, q.V, q.K, kVocabTile) || !make_tensor_map_bf16_2d(&map_w8, q.lm_head, q.V, q.K, 8) ||
-        !make_tensor_map_bf16_2d(&map_h, q.hidden, q.M, q.K, p.n_tile))
-        return cudaErrorInvalidValue;
+    CUtensorMap map_w[5], map_h;
+    for (int i = 0; i < 5; ++i)
+        if (!make_tensor_map_bf16_2d(&map_w[i], q.lm_head, q.V, q.K, kVocabTile >> i)) return cudaErrorInvalidValue;
+    if (!make_tensor_map_bf16_2d(&map_h, q.hidden, q.M, q.K, p.n_tile)) return cudaErrorInvalidValue;
 
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     cudaError_t e = cudaFuncSetAttribute(lm_head_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    lm_head_umma_kernel<<<groups * p.n_token_tiles, kThreads, smem, stream>>>(map_w128, map_w8, map_h, p);
+    lm_head_umma_kernel<<<groups * p.n_token_tiles, kThreads, smem, stream>>>(map_w[0], map_w[1], map_w[2], map_w[3], map_w[4], map_h, p);
     count_launches(1);
     return cudaGetLastError();
 }
