@@ -48,6 +48,8 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
     const float inv_T = greedy ? 1.f : 1.f / p.T;
     __shared__ Stat row_stat[kMaxRows];
     static_assert(kScanThreads / 32 >= kMaxRows, "one warp per block row");
+    pdl_wait();
+    pdl_trigger();
 
     if (warp < R) {
         const int row = b * R + warp;
@@ -181,6 +183,8 @@ __global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptP
     const int c = blockIdx.x, b = blockIdx.y, t = threadIdx.x;
     const int R = p.gamma + 1;
     const float inv_T = 1.f / p.T;
+    pdl_wait();
+    pdl_trigger();
     const SeqState st = p.seq_state[b];
     __shared__ double warp_sums[kSampleThreads / 32];
     __shared__ int s_flag;
@@ -277,6 +281,7 @@ __global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptP
 __global__ void probs_kernel(AcceptParams p) {
     const int R = p.gamma + 1, M = p.B * R;
     const int row = blockIdx.y;
+    pdl_wait();
     if (row >= M) return;
     const float inv_T = 1.f / p.T;
     __shared__ Stat red[256];
@@ -301,6 +306,7 @@ __global__ void probs_kernel(AcceptParams p) {
 
 __global__ void kv_commit_kernel(int B, int gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait();
     if (b >= B) return;
     const int a = accept_len[b];
     if (a < 1 || a > gamma + 1) { set_status(dev_status, MASSV_ERR_INVALID_ARG); return; }
@@ -310,14 +316,14 @@ __global__ void kv_commit_kernel(int B, int gamma, const int32_t* accept_len, in
 }  // namespace
 
 cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream) {
-    accept_scan_kernel<<<p.B, kScanThreads, 0, stream>>>(p);
+    if (launch_pdl(accept_scan_kernel, dim3(p.B), dim3(kScanThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
     count_launches(1);
     if (p.T > 0.f) {
-        residual_sample_kernel<<<dim3(p.n_chunks, p.B), kSampleThreads, 0, stream>>>(p);
+        if (launch_pdl(residual_sample_kernel, dim3(p.n_chunks, p.B), dim3(kSampleThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
         count_launches(1);
         if (p.probs_out) {
             const int M = p.B * (p.gamma + 1);
-            probs_kernel<<<dim3(16, M), 256, 0, stream>>>(p);
+            if (launch_pdl(probs_kernel, dim3(16, M), dim3(256), 0, stream, p) != cudaSuccess) return cudaGetLastError();
             count_launches(1);
         }
     }
@@ -327,7 +333,7 @@ cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream) {
 cudaError_t launch_kv_commit(int B, int gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
                              cudaStream_t stream) {
     if (accept_len == nullptr) return cudaSuccess;   // rollback: lengths stay
-    kv_commit_kernel<<<(B + 127) / 128, 128, 0, stream>>>(B, gamma, accept_len, seq_lens, dev_status);
+    if (launch_pdl(kv_commit_kernel, dim3((B + 127) / 128), dim3(128), 0, stream, B, gamma, accept_len, seq_lens, dev_status) != cudaSuccess) return cudaGetLastError();
     count_launches(1);
     return cudaGetLastError();
 }

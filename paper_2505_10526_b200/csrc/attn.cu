@@ -78,6 +78,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 
     const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    pdl_wait();
     const int L = p.seq_lens[b];
     if (L < 0 || L + p.R > p.max_pages * kPageSize) {            // no room for the block: skip the sequence
         if (chunk == 0 && g == 0 && threadIdx.x == 0) set_status(p.dev_status, MASSV_ERR_CAPACITY);
@@ -300,6 +301,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 
     // ---------------------------------------------------- merge the warps' partial results
     __syncthreads();                         // every tile has been consumed: the ring can be reused
+    pdl_trigger();
     float* st_o = reinterpret_cast<float*>(smem);            // [TS][RP][D]
     float* st_m = st_o + TS * RP * D;                        // [TS][RP]
     float* st_l = st_m + TS * RP;
@@ -363,6 +365,8 @@ constexpr int kCombineMaxChunks = 1024;
 __global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, int rows_pad) {
     const int G = p.Hq / p.Hkv, rows = G * p.R;
     const int r = blockIdx.x % rows, g = (blockIdx.x / rows) % p.Hkv, b = blockIdx.x / (rows * p.Hkv);
+    pdl_wait();
+    pdl_trigger();
     const int L = p.seq_lens[b];
     if (L < 0 || L + p.R > p.max_pages * kPageSize) return;
     const int n_chunks = (L + p.R + p.kv_chunk - 1) / p.kv_chunk;
@@ -413,8 +417,7 @@ cudaError_t launch_split(const AttnParams& p, const CUtensorMap& mk, const CUten
     const size_t smem = ring + (size_t)RP * D * 2 + 1024;
     cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<D, MT, TS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attn_split_kernel<D, MT, TS><<<dim3(p.max_chunks, p.Hkv, p.B), (MT * TS + 1) * 32, smem, stream>>>(mk, mv, p);
-    return cudaGetLastError();
+    return launch_pdl(attn_split_kernel<D, MT, TS>, dim3(p.max_chunks, p.Hkv, p.B), dim3((MT * TS + 1) * 32), smem, stream, mk, mv, p);
 }
 
 template <int D>
@@ -452,7 +455,8 @@ cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
     int launched = 1;
     if (p.max_chunks > 1) {
         if (p.max_chunks > kCombineMaxChunks) return cudaErrorInvalidValue;
-        attn_combine_kernel<<<p.B * p.Hkv * rows, p.d < 128 ? 64 : 128, 0, stream>>>(p, attn_rows_pad(rows));
+        e = launch_pdl(attn_combine_kernel, dim3(p.B * p.Hkv * rows), dim3(p.d < 128 ? 64 : 128), 0, stream, p, attn_rows_pad(rows));
+        if (e != cudaSuccess) return e;
         launched = 2;
     }
     count_launches(launched);

@@ -23,6 +23,29 @@ __device__ __forceinline__ float bf16_bits_to_float(uint16_t h) {
     return __uint_as_float(((uint32_t)h) << 16);
 }
 
+// Programmatic dependent launch: every kernel is launched so that it may start
+// while its predecessor in the stream drains.  pdl_wait() blocks until the
+// predecessor has completed and its writes are visible; it must run before the
+// first access to global memory.  pdl_trigger() lets the successor begin launching.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Per-sequence result of the acceptance scan, consumed by the sampling kernels.
 struct SeqState {
     int32_t n;        // index of the row the extra token is drawn from (first rejection or gamma)

@@ -268,6 +268,7 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abort_ptr = &abort_flag;
+    pdl_wait();          // everything above overlapped with the tail of the previous kernel
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -379,6 +380,7 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
 
     tc_fence_before();
     __syncthreads();
+    pdl_trigger();
     // the CTA's statistics: merge the four lane quarters (ascending rows) into one partial slot
     for (int c = threadIdx.x; c < p.n_tile; c += kThreads) {
         const int tok = tok_base + c;
@@ -460,7 +462,9 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     cudaError_t e = cudaFuncSetAttribute(lm_head_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    lm_head_umma_kernel<<<groups * p.n_token_tiles, kThreads, smem, stream>>>(map_w[0], map_w[1], map_w[2], map_w[3], map_w[4], map_h, p);
+    e = launch_pdl(lm_head_umma_kernel, dim3(groups * p.n_token_tiles), dim3(kThreads), smem, stream, map_w[0], map_w[1], map_w[2],
+                   map_w[3], map_w[4], map_h, p);
+    if (e != cudaSuccess) return e;
     count_launches(1);
     return cudaGetLastError();
 }
