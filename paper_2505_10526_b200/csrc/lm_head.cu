@@ -54,24 +54,30 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major tile of 128-byte rows, 128-byte
-// swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);   // start address
-    d |= (uint64_t)1 << 16;                         // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;               // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                         // descriptor version (sm_100)
-    d |= (uint64_t)2 << 61;                         // 128-byte swizzle
-    return d;
+// swizzle, 8-row groups 1024 bytes apart.  This is the address-independent part.
+constexpr uint64_t umma_desc_k_sw128_const() {
+    return ((uint64_t)1 << 16)                      // leading byte offset (unused for swizzled K-major)
+           | ((uint64_t)(1024 >> 4) << 32)          // stride byte offset between 8-row groups
+           | ((uint64_t)1 << 46)                    // descriptor version (sm_100)
+           | ((uint64_t)2 << 61);                   // 128-byte swizzle
 }
 
+// The descriptor's upper word is the same for every tile; the lower word holds
+// the start address, so stepping through a tile is 32-bit arithmetic.
+constexpr uint32_t kDescHi = (uint32_t)(umma_desc_k_sw128_const() >> 32);
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16); }
+
 // D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate, one CTA.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+// ACC = false overwrites D.  Descriptors are passed as (lower word, shared upper word).
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %4};\n\t"
+        "mov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(kDescHi), "r"(ACC ? 1u : 0u)
         : "memory");
 }
 // Arrive on an mbarrier once every MMA issued so far by this thread has finished.
@@ -276,18 +282,18 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             uint64_t pol_stream, pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-            uint32_t it = 0;
+            int s = 0;
+            uint32_t ph = 0;
+            uint8_t* w_dst = smem;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
                 const int v0 = row_begin + t * tile_rows;
                 const int rows = min(tile_rows, row_end - v0);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (it / p.stages) & 1u;
+                const uint32_t tx_bytes = (uint32_t)(rows * 128 + p.n_tile * 128);
+                for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_ptr)) { ok = false; break; }
-                    uint8_t* w_dst = smem + (size_t)s * stage_bytes;
                     uint8_t* h_dst = w_dst + kTileBytesW;
-                    mbar_expect_tx(&full_bar[s], (uint32_t)(rows * 128 + p.n_tile * 128));
+                    mbar_expect_tx(&full_bar[s], tx_bytes);
                     if (rows == kVocabTile) {
                         tma_load_2d(w_dst, &map_w128, kb * kBlockK, v0, &full_bar[s], pol_stream);
                     } else {
@@ -299,6 +305,8 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
                         if (rows & 8) { tma_load_2d(w_dst + r * 128, &map_w8, kb * kBlockK, v0 + r, &full_bar[s], pol_stream); r += 8; }
                     }
                     tma_load_2d(h_dst, &map_h, kb * kBlockK, tok_base, &full_bar[s], pol_keep);
+                    w_dst += stage_bytes;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; w_dst = smem; }
                 }
             }
             if (!ok) {
@@ -311,26 +319,31 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
         if (lane == 0) {
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) |
                                    ((uint32_t)(kVocabTile >> 4) << 24);
-            uint32_t it = 0;
+            // The issuing thread must stay far below the 64..128 cycles one MMA takes, so the
+            // loop carries only 32-bit descriptor words and a stage counter.
+            const uint32_t lo_step = (uint32_t)stage_bytes >> 4;
+            const uint32_t a_lo0 = umma_desc_lo(smem_u32(smem));
+            int s = 0;
+            uint32_t ph = 0, a_lo = a_lo0;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
                 const int buf = t & 1;
                 if (!mbar_wait(&tmem_empty_bar[buf], (((uint32_t)t >> 1) & 1u) ^ 1u, abort_ptr)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.n_tile);
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const int s = it % p.stages;
-                    const uint32_t ph = (it / p.stages) & 1u;
+                for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&full_bar[s], ph, abort_ptr)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
-                    const uint32_t b_addr = a_addr + kTileBytesW;
-#pragma unroll
-                    for (int k = 0; k < kBlockK / 16; ++k) {
-                        umma_bf16(d_tmem, umma_desc_k_sw128(a_addr + k * 32), umma_desc_k_sw128(b_addr + k * 32), idesc,
-                                  (kb | k) != 0 ? 1u : 0u);
-                    }
+                    const uint32_t b_lo = a_lo + (kTileBytesW >> 4);
+                    // four K slices of 16 elements (32 bytes, i.e. 2 descriptor units) each
+                    if (kb == 0) umma_bf16<false>(d_tmem, a_lo, b_lo, idesc);
+                    else umma_bf16<true>(d_tmem, a_lo, b_lo, idesc);
+                    umma_bf16<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                    umma_bf16<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                    umma_bf16<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
                     umma_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
+                    a_lo += lo_step;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; a_lo = a_lo0; }
                 }
                 if (ok) umma_commit(&tmem_full_bar[buf]);
             }
