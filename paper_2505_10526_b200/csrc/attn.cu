@@ -7,7 +7,7 @@
 // Work item = (sequence, KV head, chunk of kv_chunk positions); grid =
 // (max_chunks, Hkv, B) and CTAs whose chunk lies beyond the sequence retire at
 // once, so the hardware scheduler balances ragged lengths.  Inside a CTA a
-// producer warp streams 64-token K/V tiles page by page with TMA (16 x 64 boxes,
+// producer warp streams 64-token (32-token at d = 256) K/V tiles page by page with TMA (16 x 64 boxes,
 // 128-byte swizzle, no multicast) into an mbarrier ring; consumer warps run
 // Q K^T and P V on warp-level tensor-core MMAs (m16n8k16, bf16 -> fp32) with an
 // online softmax in registers: warp (mt, ts) owns 16 query rows and a 64/TS-token
@@ -22,7 +22,7 @@ namespace massv {
 
 namespace {
 
-constexpr int kTile = 64;            // tokens per pipeline stage
+constexpr int kChunkAlign = 64;      // kv_chunk granularity (a multiple of every tile size)
 constexpr int kMaxChunkPages = 256;  // kv_chunk <= 4096 tokens
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
@@ -51,19 +51,21 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // 128-byte rows laid out with the 128-byte swizzle (what TMA writes).
 __device__ __forceinline__ uint32_t swz(int row, int unit) { return (uint32_t)(row * 128 + ((unit ^ (row & 7)) << 4)); }
 
-template <int D>
+// TILE = tokens per pipeline stage (32 or 64).
+template <int D, int TILE>
 struct AttnCfg {
     static constexpr int kChunks = D / 64;                 // 64-element column groups of a row
-    static constexpr int kRegion = kTile * 128;            // bytes of one (64 tokens x 64 elements) region
+    static constexpr int kRegion = TILE * 128;             // bytes of one (TILE tokens x 64 elements) region
     static constexpr int kBytesK = kChunks * kRegion;
     static constexpr int kStageBytes = 2 * kBytesK;        // K then V
     static constexpr int kStages = (D == 64) ? 4 : 3;
 };
 
-template <int D, int MT, int TS>
+template <int D, int MT, int TS, int TILE>
 __global__ void __launch_bounds__((MT * TS + 1) * 32, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
-    using Cfg = AttnCfg<D>;
+    using Cfg = AttnCfg<D, TILE>;
+    constexpr int kTile = TILE;
     constexpr int NW = MT * TS;            // consumer warps
     constexpr int NT = kTile / TS;         // tokens of a tile owned by one warp
     constexpr int RP = MT * 16;            // padded query rows
@@ -408,25 +410,27 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, i
     if (p.lse && threadIdx.x == 0) p.lse[row_out] = (M + log2f(Lsum)) * 0.6931471805599453f;
 }
 
-template <int D, int MT, int TS>
+template <int D, int MT, int TS, int TILE>
 cudaError_t launch_split(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream) {
-    using Cfg = AttnCfg<D>;
+    using Cfg = AttnCfg<D, TILE>;
     constexpr int RP = MT * 16;
     const size_t ring = (size_t)Cfg::kStages * Cfg::kStageBytes;
     static_assert((size_t)TS * RP * D * 4 + 2 * TS * RP * 4 <= (size_t)Cfg::kStages * Cfg::kStageBytes, "merge staging fits the ring");
     const size_t smem = ring + (size_t)RP * D * 2 + 1024;
-    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<D, MT, TS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(attn_split_kernel<D, MT, TS, TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_split_kernel<D, MT, TS>, dim3(p.max_chunks, p.Hkv, p.B), dim3((MT * TS + 1) * 32), smem, stream, mk, mv, p);
+    return launch_pdl(attn_split_kernel<D, MT, TS, TILE>, dim3(p.max_chunks, p.Hkv, p.B), dim3((MT * TS + 1) * 32), smem, stream, mk, mv, p);
 }
 
 template <int D>
 cudaError_t launch_split_d(const AttnParams& p, int mt, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream) {
     switch (mt) {
-        case 1: return launch_split<D, 1, 4>(p, mk, mv, stream);
-        case 2: return launch_split<D, 2, 2>(p, mk, mv, stream);
-        case 3: return launch_split<D, 3, 1>(p, mk, mv, stream);
-        case 4: return launch_split<D, 4, 1>(p, mk, mv, stream);
+        // d = 256 uses 32-token stages so that two CTAs (three 32 KB stages each) share an SM and
+        // one CTA's set-up and merge overlap the other's streaming
+        case 1: return D == 256 ? launch_split<D, 1, 2, 32>(p, mk, mv, stream) : launch_split<D, 1, 4, 64>(p, mk, mv, stream);
+        case 2: return D == 256 ? launch_split<D, 2, 2, 32>(p, mk, mv, stream) : launch_split<D, 2, 2, 64>(p, mk, mv, stream);
+        case 3: return D == 256 ? launch_split<D, 3, 1, 32>(p, mk, mv, stream) : launch_split<D, 3, 1, 64>(p, mk, mv, stream);
+        case 4: return D == 256 ? launch_split<D, 4, 1, 32>(p, mk, mv, stream) : launch_split<D, 4, 1, 64>(p, mk, mv, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -436,7 +440,7 @@ cudaError_t launch_split_d(const AttnParams& p, int mt, const CUtensorMap& mk, c
 int attn_rows_pad(int group_rows) { return (group_rows + 15) / 16 * 16; }
 
 cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
-    if (p.kv_chunk % kTile != 0 || p.kv_chunk > kMaxChunkPages * kPageSize) return cudaErrorInvalidValue;
+    if (p.kv_chunk % kChunkAlign != 0 || p.kv_chunk > kMaxChunkPages * kPageSize) return cudaErrorInvalidValue;
     CUtensorMap mk, mv;
     const uint64_t rows_total = (uint64_t)p.num_pages * p.Hkv * kPageSize;
     if (!make_tensor_map_bf16_2d(&mk, p.k_pages, rows_total, p.d, kPageSize) ||
