@@ -20,11 +20,14 @@ constexpr size_t kAlign = 256;
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int auto_kv_chunk(const massv_attn_desc& d) {
-    // Aim at roughly four resident work items per SM over the longest context
-    // the page table can describe; never split finer than 64 tokens.
-    const double tokens = (double)d.batch * d.max_pages_per_seq * kPageSize * d.n_kv_heads;
-    long chunk = (long)ceil(tokens / (148.0 * 4.0));
-    chunk = (chunk + 63) / 64 * 64;
+    // Work is counted in token-heads over the longest context the page table can describe.
+    // Large problems: about five waves of CTAs (two per SM), but chunks of at least 768 tokens
+    // so that the partial results written per chunk stay a few percent of the K/V read.
+    // Small problems (too few CTAs that way): split down to 64 tokens to fill the machine.
+    const double th = (double)d.batch * d.max_pages_per_seq * kPageSize * d.n_kv_heads;
+    long chunk = ((long)ceil(th / 1480.0) + 63) / 64 * 64;
+    if (chunk < 768) chunk = 768;
+    if (th / (double)chunk < 128.0) chunk = ((long)ceil(th / 128.0) + 63) / 64 * 64;
     if (chunk < 64) chunk = 64;
     if (chunk > 4096) chunk = 4096;
     return (int)chunk;

@@ -51,20 +51,24 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // 128-byte rows laid out with the 128-byte swizzle (what TMA writes).
 __device__ __forceinline__ uint32_t swz(int row, int unit) { return (uint32_t)(row * 128 + ((unit ^ (row & 7)) << 4)); }
 
-// TILE = tokens per pipeline stage (32 or 64).
-template <int D, int TILE>
+// TILE = tokens per pipeline stage (32 or 64).  DEEP: the CTA has an SM to itself (five
+// warps), so the ring is twice as deep to keep enough bytes in flight.
+template <int D, int TILE, bool DEEP>
 struct AttnCfg {
     static constexpr int kChunks = D / 64;                 // 64-element column groups of a row
     static constexpr int kRegion = TILE * 128;             // bytes of one (TILE tokens x 64 elements) region
     static constexpr int kBytesK = kChunks * kRegion;
     static constexpr int kStageBytes = 2 * kBytesK;        // K then V
-    static constexpr int kStages = (D == 64) ? 4 : 3;
+    static constexpr int kStages = DEEP ? 6 : ((D == 64) ? 4 : 3);
 };
 
+// Two CTAs should share an SM (one CTA's set-up and merge hide behind the other's
+// streaming).  Each scheduler owns a quarter of the register file and a CTA's warps are
+// dealt round-robin, so that needs at most four warps per CTA, producer included.
 template <int D, int MT, int TS, int TILE>
-__global__ void __launch_bounds__((MT * TS + 1) * 32, 1)
+__global__ void __launch_bounds__((MT * TS + 1) * 32, (MT * TS + 1) <= 4 ? 2 : 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
-    using Cfg = AttnCfg<D, TILE>;
+    using Cfg = AttnCfg<D, TILE, (MT * TS + 1 > 4)>;
     constexpr int kTile = TILE;
     constexpr int NW = MT * TS;            // consumer warps
     constexpr int NT = kTile / TS;         // tokens of a tile owned by one warp
@@ -412,7 +416,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, i
 
 template <int D, int MT, int TS, int TILE>
 cudaError_t launch_split(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream) {
-    using Cfg = AttnCfg<D, TILE>;
+    using Cfg = AttnCfg<D, TILE, (MT * TS + 1 > 4)>;
     constexpr int RP = MT * 16;
     const size_t ring = (size_t)Cfg::kStages * Cfg::kStageBytes;
     static_assert((size_t)TS * RP * D * 4 + 2 * TS * RP * 4 <= (size_t)Cfg::kStages * Cfg::kStageBytes, "merge staging fits the ring");
@@ -427,8 +431,8 @@ cudaError_t launch_split_d(const AttnParams& p, int mt, const CUtensorMap& mk, c
     switch (mt) {
         // d = 256 uses 32-token stages so that two CTAs (three 32 KB stages each) share an SM and
         // one CTA's set-up and merge overlap the other's streaming
-        case 1: return D == 256 ? launch_split<D, 1, 2, 32>(p, mk, mv, stream) : launch_split<D, 1, 4, 64>(p, mk, mv, stream);
-        case 2: return D == 256 ? launch_split<D, 2, 2, 32>(p, mk, mv, stream) : launch_split<D, 2, 2, 64>(p, mk, mv, stream);
+        case 1: return D == 256 ? launch_split<D, 1, 2, 32>(p, mk, mv, stream) : launch_split<D, 1, 2, 64>(p, mk, mv, stream);
+        case 2: return D == 256 ? launch_split<D, 2, 1, 32>(p, mk, mv, stream) : launch_split<D, 2, 1, 64>(p, mk, mv, stream);
         case 3: return D == 256 ? launch_split<D, 3, 1, 32>(p, mk, mv, stream) : launch_split<D, 3, 1, 64>(p, mk, mv, stream);
         case 4: return D == 256 ? launch_split<D, 4, 1, 32>(p, mk, mv, stream) : launch_split<D, 4, 1, 64>(p, mk, mv, stream);
         default: return cudaErrorInvalidValue;
