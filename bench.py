@@ -254,11 +254,8 @@ def main():
     t_accept = sum(e[1].elapsed_time(e[2]) for e in split_ev) / len(split_ev)
     t_commit = sum(e[2].elapsed_time(e[3]) for e in split_ev) / len(split_ev)
     t_step = sum(e[0].elapsed_time(e[3]) for e in events) / K        # ms on the device, per step
-    t_max = torch.tensor([t_step], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
-    ms_per_step = float(t_max.item())
-    value = world * cfg.m / (ms_per_step * 1e-3)
+    from paper_2505_10526_b200.replicas import aggregate_throughput
+    ms_per_step, value = aggregate_throughput(cfg.m, t_step, dev)
     assert int(step.dev_status.item()) == 0, "device-side error during the timed region"
 
     # ---- end to end: per-step inputs start in pinned host memory, results end there
@@ -277,9 +274,7 @@ def main():
         e2e_t += time.perf_counter() - t0
         between_steps()
         torch.cuda.synchronize()
-    e2e_ms = torch.tensor([e2e_t / Ke * 1e3], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_ms_per_step, e2e_value = aggregate_throughput(cfg.m, e2e_t / Ke * 1e3, dev)
     h2d, d2h = step.host_bytes_per_step(host_inputs)
 
     if rank != 0:
@@ -317,7 +312,7 @@ def main():
                      "frac": attn_bytes / (t_attn * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "mean_accept_len": float(step.accept_len.float().mean()),
         "roofline": roofline, "clocks": clocks,
-        "e2e": {"value": world * cfg.m / (float(e2e_ms.item()) * 1e-3), "unit": UNIT, "ms_per_step": float(e2e_ms.item()),
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms_per_step,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches), "wall_s_timed_region": wall,
     }
