@@ -31,6 +31,9 @@ UNIT = "positions/s"
 DEFAULT_WORKLOAD = "qwen7b_b1_t0"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 L2_FLUSH_BYTES = 512 << 20
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (per workload; None where no capture of the current kernel exists)
+NCU_TRAFFIC_BYTES = {"qwen7b_b1_t0": 1.090107e9 + 3.543e6}
 
 
 def load_peaks():
@@ -295,7 +298,8 @@ def main():
                     "achieved": lm_bytes / (t_accept * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
     roofline["frac"] = roofline["achieved"] / roofline["peak"]
     roofline["peak_source"] = f"of {peak_src}"
-    roofline["traffic"] = None
+    roofline["traffic"] = NCU_TRAFFIC_BYTES.get(cfg.name)
+    roofline["algorithmic"] = lm_bytes if roofline["bound"] == "hbm" else lm_flops
     roofline["ms_per_launch"] = t_accept
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
