@@ -34,13 +34,13 @@ def _report(entry):
     print(entry)
 
 
-def run_case(name, subset=None, check_determinism=True):
+def run_case(name, subset=None, check_determinism=True, cfg=None, **step_kw):
     from paper_2505_10526_b200 import VerifyStep
-    cfg = get_config(name)
+    cfg = cfg or get_config(name)
     w = generate(cfg, device="cuda")
     pools_before = (w["k_pages"].clone(), w["v_pages"].clone())
     seq_before = w["seq_lens"].clone()
-    step = VerifyStep.for_workload(cfg, w, want_logits=True, want_probs=True, want_attn_f32=True)
+    step = VerifyStep.for_workload(cfg, w, want_logits=True, want_probs=True, want_attn_f32=True, **step_kw)
     step.run(w, commit=True)
     torch.cuda.synchronize()
     assert int(step.dev_status.item()) == 0
@@ -190,3 +190,30 @@ def test_gamma_zero_is_plain_decoding():
     torch.cuda.synchronize()
     st = compare_accept(ref, step.out_tokens.cpu().numpy(), step.accept_len.cpu().numpy(), 0)
     assert st["hard"] == 0 and np.all(step.accept_len.cpu().numpy() == 1)
+
+
+ODD_SHAPES = [
+    # vocabulary not a multiple of the 128-row tile, hidden = 5 K-blocks, 7 rows per sequence
+    dict(name="odd_vocab_t1", batch=3, gamma=6, n_q_heads=4, n_kv_heads=2, head_dim=64, hidden=320, vocab=1160,
+         temperature=0.8, ctx_lo=0, ctx_hi=150),
+    dict(name="odd_vocab_t0", batch=2, gamma=2, n_q_heads=2, n_kv_heads=2, head_dim=128, hidden=192, vocab=8200,
+         temperature=0.0, ctx_lo=1, ctx_hi=70),
+    # 8 query heads per KV head and gamma = 7: 64 query rows per CTA (four MMA row tiles), d = 256
+    dict(name="wide_group_d256", batch=2, gamma=7, n_q_heads=8, n_kv_heads=1, head_dim=256, hidden=256, vocab=1024,
+         temperature=1.0, ctx_lo=100, ctx_hi=400),
+    # d = 256 with three row tiles, and d = 64 with one
+    dict(name="three_tiles_d256", batch=2, gamma=5, n_q_heads=14, n_kv_heads=2, head_dim=256, hidden=256, vocab=1024,
+         temperature=0.0, ctx_lo=60, ctx_hi=260),
+    dict(name="one_tile_d64", batch=5, gamma=1, n_q_heads=6, n_kv_heads=3, head_dim=64, hidden=128, vocab=512,
+         temperature=1.3, ctx_lo=0, ctx_hi=500),
+]
+
+
+@pytest.mark.parametrize("spec", ODD_SHAPES, ids=[s["name"] for s in ODD_SHAPES])
+@pytest.mark.parametrize("kv_chunk", [0, 64])
+def test_odd_shapes_and_forced_splits(spec, kv_chunk):
+    """Shapes off the benchmark grid (ragged vocabulary tile, every MMA row-tile count, all head
+    dims), with the automatic chunking and with 64-token chunks that force the merge kernel."""
+    from workloads import VerifyConfig
+    cfg = VerifyConfig(image_tokens=0.25, draft_noise_std=0.7, seed=40 + len(spec["name"]), **spec)
+    run_case(None, cfg=cfg, kv_chunk=kv_chunk)
