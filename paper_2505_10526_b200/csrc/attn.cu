@@ -132,33 +132,34 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
 
     if (warp == NW) {
         // ------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint64_t policy;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-            for (int t = 0; t < n_tiles; ++t) {
-                const int s = t % Cfg::kStages;
-                const uint32_t ph = ((uint32_t)(t / Cfg::kStages)) & 1u;
-                if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_ptr)) break;
-                const int tile_start = c_begin + t * kTile;
-                int n_pg = (c_end - tile_start + kPageSize - 1) / kPageSize;
-                if (n_pg > kTile / kPageSize) n_pg = kTile / kPageSize;
-                uint8_t* kdst = smem + (size_t)s * Cfg::kStageBytes;
-                uint8_t* vdst = kdst + Cfg::kBytesK;
-                mbar_expect_tx(&full_bar[s], (uint32_t)(n_pg * NCH * 2048 * 2));
-                for (int pg = 0; pg < n_pg; ++pg) {
-                    int pid = s_pages[t * (kTile / kPageSize) + pg];
-                    if (pid < 0 || pid >= p.num_pages) { set_status(p.dev_status, MASSV_ERR_CAPACITY); pid = 0; }
-                    const int row = (pid * p.Hkv + g) * kPageSize;
-#pragma unroll
-                    for (int dc = 0; dc < NCH; ++dc) {
-                        tma_load_2d(kdst + dc * Cfg::kRegion + pg * 2048, &map_k, dc * 64, row, &full_bar[s], policy);
-                        tma_load_2d(vdst + dc * Cfg::kRegion + pg * 2048, &map_v, dc * 64, row, &full_bar[s], policy);
-                    }
-                }
+        // A tile is 2 * (d/64) boxes per page.  One box per lane: a single thread issuing them one
+        // after the other cannot keep an SM's share of HBM busy when the CTA has the SM to itself.
+        uint64_t policy;
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+        for (int t = 0; t < n_tiles; ++t) {
+            const int s = t % Cfg::kStages;
+            const uint32_t ph = ((uint32_t)(t / Cfg::kStages)) & 1u;
+            int freed = 0;
+            if (lane == 0) freed = mbar_wait(&empty_bar[s], ph ^ 1u, abort_ptr) ? 1 : 0;
+            freed = __shfl_sync(0xffffffffu, freed, 0);
+            if (!freed) break;
+            const int tile_start = c_begin + t * kTile;
+            int n_pg = (c_end - tile_start + kPageSize - 1) / kPageSize;
+            if (n_pg > kTile / kPageSize) n_pg = kTile / kPageSize;
+            uint8_t* kdst = smem + (size_t)s * Cfg::kStageBytes;
+            if (lane == 0) mbar_expect_tx(&full_bar[s], (uint32_t)(n_pg * NCH * 2048 * 2));
+            __syncwarp();
+            for (int i = lane; i < n_pg * NCH * 2; i += 32) {
+                const int is_v = i & 1, dc = (i >> 1) % NCH, pg = i / (2 * NCH);
+                int pid = s_pages[t * (kTile / kPageSize) + pg];
+                if (pid < 0 || pid >= p.num_pages) { set_status(p.dev_status, MASSV_ERR_CAPACITY); pid = 0; }
+                const int row = (pid * p.Hkv + g) * kPageSize;
+                tma_load_2d(kdst + is_v * Cfg::kBytesK + dc * Cfg::kRegion + pg * 2048, is_v ? &map_v : &map_k, dc * 64, row,
+                            &full_bar[s], policy);
             }
-            if (*abort_ptr) {
-                for (int i = 0; i < 64; ++i) __nanosleep(2000);   // let copies in flight land
-            }
+        }
+        if (lane == 0 && *abort_ptr) {
+            for (int i = 0; i < 64; ++i) __nanosleep(2000);   // let copies in flight land
         }
     } else {
         // ------------------------------------------------ consumers

@@ -87,6 +87,11 @@ _add(VerifyConfig("tiny_ragged_t0", 5, 7, **_TINY, temperature=0.0, ctx_lo=0, ct
 _add(replace(CONFIGS["qwen7b_b16_t1"], name="qwen7b_b16_t1_peaked", hidden_std=5.0, seed=13))
 
 
+# Reduced-batch copies of the long-context points, small enough for multi-pass profiler captures.
+for _g in (5, 7):
+    _add(replace(CONFIGS[f"qwen7b_long_g{_g}_t0"], name=f"qwen7b_long_b16_g{_g}_t0", batch=16))
+
+
 def get_config(name: str) -> VerifyConfig:
     if name not in CONFIGS:
         raise KeyError(f"unknown workload {name!r}; known: {sorted(CONFIGS)}")
