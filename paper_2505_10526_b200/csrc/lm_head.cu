@@ -32,6 +32,7 @@ constexpr int kTileBytesW = kVocabTile * kBlockK * 2;
 constexpr int kMaxStages = 12;
 constexpr int kMaxCtas = 192;               // partial slots are sized for at most this many CTAs
 constexpr int kRingBytes = 200 * 1024;      // shared memory given to the TMA ring
+constexpr int kPairMinTile = 64;            // token rows per tile from which CTA pairs are used
 
 struct UmmaParams {
     int M, K, V;
@@ -83,6 +84,52 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32
 // Arrive on an mbarrier once every MMA issued so far by this thread has finished.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// ---- CTA pairs (cta_group::2): two CTAs of a cluster act as one 256-row MMA.  Each loads its own
+// 128 weight rows and half of the hidden-state rows; the even CTA (the leader) issues the MMAs,
+// which read both CTAs' shared memory and write each CTA's half of the result to its own TMEM.
+__device__ __forceinline__ uint32_t cluster_cta_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Cluster-wide address of a shared-memory location in CTA `rank`.
+__device__ __forceinline__ uint32_t cluster_addr(const void* local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(local)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_expect_tx_at(uint32_t bar_cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_at(uint32_t bar_cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// TMA load into this CTA's shared memory whose completion is signalled on a barrier of the pair's leader.
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster_addr,
+                                                 uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(smem_u32(dst)),
+        "l"(map), "r"(x), "r"(y), "r"(bar_cluster_addr), "l"(policy)
+        : "memory");
+}
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %4};\n\t"
+        "mov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(kDescHi), "r"(ACC ? 1u : 0u)
+        : "memory");
+}
+// Arrive, in both CTAs of the pair, on the barrier at this shared-memory offset once the MMAs issued so far are done.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
+                 "h"((uint16_t)3)
+                 : "memory");
 }
 
 template <int C>
@@ -225,6 +272,10 @@ __device__ __forceinline__ void drain_chunk(const UmmaParams& p, uint32_t taddr,
     running = stat_combine(running, mine, p.scale_log2, greedy);
 }
 
+// PAIR: the grid is made of 2-CTA clusters; a pair works on 256-row vocabulary super-tiles (CTA rank r
+// owns rows 128 r .. 128 r + 127 and half of the token rows of the hidden-state tile), which halves the
+// hidden-state traffic per weight byte compared with one CTA per 128 rows.
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_constant__ CUtensorMap map_w64,
                     const __grid_constant__ CUtensorMap map_w32, const __grid_constant__ CUtensorMap map_w16,
@@ -243,34 +294,46 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const int stage_bytes = kTileBytesW + p.n_tile * 128;
+    const int h_rows = PAIR ? p.n_tile / 2 : p.n_tile;       // hidden-state rows this CTA loads per K block
+    const int stage_bytes = kTileBytesW + h_rows * 128;
     const int num_kb = p.K / kBlockK;
+    const uint32_t pair_rank = PAIR ? cluster_cta_rank() : 0u;
 
-    // which band of vocabulary rows and which token tile this CTA owns
-    const int group = blockIdx.x / p.n_token_tiles;
-    const int token_tile = blockIdx.x % p.n_token_tiles;
-    const int row_begin = min(p.V, group * p.tiles_per_group * kVocabTile);
-    const int row_end = min(p.V, row_begin + p.tiles_per_group * kVocabTile);
-    constexpr int tile_rows = kVocabTile;
+    // which band of vocabulary rows and which token tile this CTA (or pair) owns
+    const int unit = PAIR ? blockIdx.x / 2 : blockIdx.x;
+    const int group = unit / p.n_token_tiles;
+    const int token_tile = unit % p.n_token_tiles;
+    constexpr int tile_rows = PAIR ? 2 * kVocabTile : kVocabTile;       // rows per (super-)tile of the band
+    const int row_begin = min(p.V, group * p.tiles_per_group * tile_rows);
+    const int row_end = min(p.V, row_begin + p.tiles_per_group * tile_rows);
     const int n_tiles = (row_end - row_begin + tile_rows - 1) / tile_rows;
     const int tok_base = token_tile * p.n_tile;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], kEpilogueWarps); }
+        // in a pair the leader's tmem_empty barriers collect both CTAs' epilogue warps
+        for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], (PAIR ? 2 : 1) * kEpilogueWarps); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
         __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                     "r"((uint32_t)p.tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if constexpr (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                         "r"((uint32_t)p.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                         "r"((uint32_t)p.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();      // the peer's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abort_ptr = &abort_flag;
@@ -287,12 +350,24 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             uint8_t* w_dst = smem;
             bool ok = true;
             for (int t = 0; t < n_tiles && ok; ++t) {
-                const int v0 = row_begin + t * tile_rows;
-                const int rows = min(tile_rows, row_end - v0);
+                const int v0 = row_begin + t * tile_rows + (int)pair_rank * kVocabTile;
+                const int rows = PAIR ? kVocabTile : min(tile_rows, row_end - v0);
                 const uint32_t tx_bytes = (uint32_t)(rows * 128 + p.n_tile * 128);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_ptr)) { ok = false; break; }
                     uint8_t* h_dst = w_dst + kTileBytesW;
+                    if constexpr (PAIR) {
+                        // Both CTAs' copies complete on the leader's barrier; the leader announces the
+                        // bytes of the pair (two 128-row weight boxes, two halves of the hidden-state tile;
+                        // rows past the end of either matrix are filled with zeros and still counted).
+                        const uint32_t bar = cluster_addr(&full_bar[s], 0);
+                        if (pair_rank == 0) mbar_expect_tx_at(bar, (uint32_t)(2 * kTileBytesW + p.n_tile * 128));
+                        tma_load_2d_pair(w_dst, &map_w128, kb * kBlockK, v0, bar, pol_stream);
+                        tma_load_2d_pair(h_dst, &map_h, kb * kBlockK, tok_base + (int)pair_rank * h_rows, bar, pol_keep);
+                        w_dst += stage_bytes;
+                        if (++s == p.stages) { s = 0; ph ^= 1u; w_dst = smem; }
+                        continue;
+                    }
                     mbar_expect_tx(&full_bar[s], tx_bytes);
                     if (rows == kVocabTile) {
                         tma_load_2d(w_dst, &map_w128, kb * kBlockK, v0, &full_bar[s], pol_stream);
@@ -316,9 +391,9 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && pair_rank == 0) {       // in a pair only the leader issues
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_tile >> 3) << 17) |
-                                   ((uint32_t)(kVocabTile >> 4) << 24);
+                                   ((uint32_t)((PAIR ? 2 * kVocabTile : kVocabTile) >> 4) << 24);
             // The issuing thread must stay far below the 64..128 cycles one MMA takes, so the
             // loop carries only 32-bit descriptor words and a stage counter.
             const uint32_t lo_step = (uint32_t)stage_bytes >> 4;
@@ -336,16 +411,28 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
                     tc_fence_after();
                     const uint32_t b_lo = a_lo + (kTileBytesW >> 4);
                     // four K slices of 16 elements (32 bytes, i.e. 2 descriptor units) each
-                    if (kb == 0) umma_bf16<false>(d_tmem, a_lo, b_lo, idesc);
-                    else umma_bf16<true>(d_tmem, a_lo, b_lo, idesc);
-                    umma_bf16<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
-                    umma_bf16<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
-                    umma_bf16<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
-                    umma_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
+                    if constexpr (PAIR) {
+                        if (kb == 0) umma_bf16_pair<false>(d_tmem, a_lo, b_lo, idesc);
+                        else umma_bf16_pair<true>(d_tmem, a_lo, b_lo, idesc);
+                        umma_bf16_pair<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                        umma_bf16_pair<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                        umma_bf16_pair<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
+                        umma_commit_pair(&empty_bar[s]);     // frees the stage in both CTAs
+                    } else {
+                        if (kb == 0) umma_bf16<false>(d_tmem, a_lo, b_lo, idesc);
+                        else umma_bf16<true>(d_tmem, a_lo, b_lo, idesc);
+                        umma_bf16<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                        umma_bf16<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                        umma_bf16<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
+                        umma_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
+                    }
                     a_lo += lo_step;
                     if (++s == p.stages) { s = 0; ph ^= 1u; a_lo = a_lo0; }
                 }
-                if (ok) umma_commit(&tmem_full_bar[buf]);
+                if (ok) {
+                    if constexpr (PAIR) umma_commit_pair(&tmem_full_bar[buf]);
+                    else umma_commit(&tmem_full_bar[buf]);
+                }
             }
         }
     } else {
@@ -367,8 +454,8 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             if (!mbar_wait(&tmem_full_bar[buf], ((uint32_t)t >> 1) & 1u, abort_ptr)) { ok = false; break; }
             tc_fence_after();
             TileCtx tile;
-            tile.v0 = row_begin + t * tile_rows;
-            tile.rows = min(tile_rows, row_end - tile.v0);
+            tile.v0 = row_begin + t * tile_rows + (int)pair_rank * kVocabTile;     // this CTA's 128 rows
+            tile.rows = max(0, min(kVocabTile, row_end - tile.v0));
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.n_tile);
             for (int c = half; c < n_chunks32; c += 2) {
                 const int col = c * 32 + lane;
@@ -387,7 +474,10 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tmem_empty_bar[buf]);
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_at(cluster_addr(&tmem_empty_bar[buf], 0));   // the leader waits for both CTAs
+                else mbar_arrive(&tmem_empty_bar[buf]);
+            }
         }
     }
 
@@ -402,16 +492,20 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
 #pragma unroll
             for (int qd = 1; qd < 4; ++qd)
                 acc = stat_combine(acc, Stat{run_m[qd][c], run_s[qd][c], run_i[qd][c]}, p.scale_log2, p.greedy != 0);
-            const size_t slot = (size_t)group * p.M;
+            const size_t slot = (size_t)(PAIR ? group * 2 + (int)pair_rank : group) * p.M;
             p.part_max[slot + tok] = acc.m;
             p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
             p.part_idx[slot + tok] = acc.idx;
         }
     }
+    if constexpr (PAIR) cluster_sync_all();      // neither CTA frees TMEM or leaves while the other may still use it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+        if constexpr (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
     }
     if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
 }
@@ -431,8 +525,8 @@ int sm_count() {
 // Upper bound of the partial slots the acceptance kernel may have to merge: one per CTA.
 int lm_head_num_partials(int M, int V) {
     (void)M;
-    const int bands = (V + kVocabTile - 1) / kVocabTile;
-    return bands < kMaxCtas ? bands : kMaxCtas;
+    const int slots = 2 * ((V + 2 * kVocabTile - 1) / (2 * kVocabTile));     // CTA pairs cover 256 rows at a time
+    return slots < kMaxCtas ? slots : kMaxCtas;
 }
 
 cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_part_used) {
@@ -443,16 +537,21 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.n_tile = (per_tile + 15) / 16 * 16;
     int ctas = sm_count();
     if (ctas > kMaxCtas) ctas = kMaxCtas;
-    // Whole tiles per CTA: a band with a short tail tile would run a full K loop with almost
+    // From 64 token rows up, pairs of CTAs (cta_group::2) share the hidden-state tile: the traffic
+    // from L2 into shared memory per weight byte drops from 1 + N/128 to 1 + N/256.
+    const bool pair = p.n_tile >= kPairMinTile;
+    const int band_rows = pair ? 2 * kVocabTile : kVocabTile;
+    // Whole tiles per CTA (pair): a band with a short tail tile would run a full K loop with almost
     // nothing in flight.  Use the fewest CTAs that still reach the minimal tiles-per-CTA count
     // (1188 tiles on 148 SMs: 132 CTAs x 9 tiles).
-    int groups = ctas / p.n_token_tiles;
-    const int bands = (q.V + kVocabTile - 1) / kVocabTile;
+    int groups = ctas / (p.n_token_tiles * (pair ? 2 : 1));
+    const int bands = (q.V + band_rows - 1) / band_rows;
     if (groups > bands) groups = bands;
     p.tiles_per_group = (bands + groups - 1) / groups;
     groups = (bands + p.tiles_per_group - 1) / p.tiles_per_group;
     p.n_groups = groups;
-    const int stage_bytes = kTileBytesW + p.n_tile * 128;
+    const int h_rows = pair ? p.n_tile / 2 : p.n_tile;
+    const int stage_bytes = kTileBytesW + h_rows * 128;
     int stages = kRingBytes / stage_bytes;
     if (stages > kMaxStages) stages = kMaxStages;
     p.stages = stages;
@@ -464,19 +563,28 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.logits = q.logits;
     p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
     p.dev_status = q.dev_status;
-    if (groups > q.n_part) return cudaErrorInvalidValue;
-    *n_part_used = groups;
+    const int slots = groups * (pair ? 2 : 1);
+    if (slots > q.n_part) return cudaErrorInvalidValue;
+    *n_part_used = slots;
 
     CUtensorMap map_w[5], map_h;
     for (int i = 0; i < 5; ++i)
         if (!make_tensor_map_bf16_2d(&map_w[i], q.lm_head, q.V, q.K, kVocabTile >> i)) return cudaErrorInvalidValue;
-    if (!make_tensor_map_bf16_2d(&map_h, q.hidden, q.M, q.K, p.n_tile)) return cudaErrorInvalidValue;
+    if (!make_tensor_map_bf16_2d(&map_h, q.hidden, q.M, q.K, h_rows)) return cudaErrorInvalidValue;
 
     const size_t smem = (size_t)stages * stage_bytes + 1024;
-    cudaError_t e = cudaFuncSetAttribute(lm_head_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(lm_head_umma_kernel, dim3(groups * p.n_token_tiles), dim3(kThreads), smem, stream, map_w[0], map_w[1], map_w[2],
-                   map_w[3], map_w[4], map_h, p);
+    cudaError_t e;
+    if (pair) {
+        e = cudaFuncSetAttribute(lm_head_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        e = launch_pdl_cluster(lm_head_umma_kernel<true>, dim3(groups * p.n_token_tiles * 2), dim3(kThreads), smem, stream, 2,
+                               map_w[0], map_w[1], map_w[2], map_w[3], map_w[4], map_h, p);
+    } else {
+        e = cudaFuncSetAttribute(lm_head_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        e = launch_pdl(lm_head_umma_kernel<false>, dim3(groups * p.n_token_tiles), dim3(kThreads), smem, stream, map_w[0],
+                       map_w[1], map_w[2], map_w[3], map_w[4], map_h, p);
+    }
     if (e != cudaSuccess) return e;
     count_launches(1);
     return cudaGetLastError();
