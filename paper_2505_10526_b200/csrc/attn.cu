@@ -8,7 +8,7 @@
 // (max_chunks, Hkv, B) and CTAs whose chunk lies beyond the sequence retire at
 // once, so the hardware scheduler balances ragged lengths.  Inside a CTA a
 // producer warp streams 64-token (32-token at d = 256) K/V tiles page by page with TMA (16 x 64 boxes,
-// 128-byte swizzle, no multicast) into an mbarrier ring; consumer warps run
+// 128-byte swizzle) into an mbarrier ring; consumer warps run
 // Q K^T and P V on warp-level tensor-core MMAs (m16n8k16, bf16 -> fp32) with an
 // online softmax in registers: warp (mt, ts) owns 16 query rows and a 64/TS-token
 // slice of every tile.  Partial (max, sum, O) of the warps are merged through
