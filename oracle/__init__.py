@@ -62,15 +62,16 @@ def kv_append(k_new, v_new, k_pages, v_pages, page_table, seq_lens):
                              _p(page_table, np.int32), _p(seq_lens, np.int32))
 
 
-def verify_attn(q, k_pages, v_pages, page_table, seq_lens, scale=None):
-    """Block attention over the (already appended) cache. Returns (out f64 [B,R,Hq,d], lse f64 [B,R,Hq])."""
+def verify_attn(q, k_pages, v_pages, page_table, seq_lens, scale=None, window=0):
+    """Block attention over the (already appended) cache. Returns (out f64 [B,R,Hq,d], lse f64 [B,R,Hq]).
+    window > 0: each row sees only the last `window` positions up to itself."""
     B, R, Hq, d = q.shape
     Hkv, page = k_pages.shape[1], k_pages.shape[2]
     if scale is None:
         scale = 1.0 / np.sqrt(d)
     out = np.zeros((B, R, Hq, d), dtype=np.float64)
     lse = np.zeros((B, R, Hq), dtype=np.float64)
-    _load().oracle_verify_attn(B, R, Hq, Hkv, d, page, page_table.shape[1], ctypes.c_double(scale),
+    _load().oracle_verify_attn(B, R, Hq, Hkv, d, page, page_table.shape[1], int(window), ctypes.c_double(scale),
                                _p(q, np.uint16), _p(k_pages, np.uint16), _p(v_pages, np.uint16),
                                _p(page_table, np.int32), _p(seq_lens, np.int32), _p(out, np.float64), _p(lse, np.float64))
     return out, lse
@@ -122,7 +123,7 @@ def tvd(p, q):
     return float(_load().oracle_tvd(p.shape[0], _p(p, np.float64), _p(q, np.float64)))
 
 
-def verify_step(w, temperature, scale=None, want_attention=True):
+def verify_step(w, temperature, scale=None, want_attention=True, window=0):
     """Whole verify step on a workload dict of torch tensors (see ``workloads.generate``).
 
     Returns a dict with numpy results; the workload's page pools are not modified
@@ -134,7 +135,7 @@ def verify_step(w, temperature, scale=None, want_attention=True):
         kp, vp = bf16_bits(w["k_pages"]).copy(), bf16_bits(w["v_pages"]).copy()
         pt = w["page_table"].cpu().numpy().astype(np.int32)
         kv_append(bf16_bits(w["k_new"]), bf16_bits(w["v_new"]), kp, vp, pt, seq)
-        res["attn_out"], res["lse"] = verify_attn(bf16_bits(w["q"]), kp, vp, pt, seq, scale)
+        res["attn_out"], res["lse"] = verify_attn(bf16_bits(w["q"]), kp, vp, pt, seq, scale, window)
         res["k_pages"], res["v_pages"] = kp, vp
     B, R, K = w["hidden"].shape
     z = logits(bf16_bits(w["hidden"]).reshape(B * R, K), bf16_bits(w["lm_head"]))

@@ -70,9 +70,14 @@ void oracle_kv_append(int B, int R, int n_kv_heads, int head_dim, int page_size,
  *   out[b,j,h,:] = sum_i softmax_i(scale * <q[b,j,h,:], K[i]>) * V[i]
  *   lse[b,j,h]   = log sum_i exp(scale * <q, K[i]>)
  * The block must already be appended.  q : bf16 [B,R,Hq,d]; out : f64 same shape.
+ *
+ * window > 0 selects sliding-window attention (the local layers of Gemma3-style
+ * targets, which the paper's Sec. 4 notes as an architectural difference without
+ * fixing a size): the row at position P sees only positions P-window+1 .. P.
+ * window == 0 is full attention.
  */
 void oracle_verify_attn(int B, int R, int n_q_heads, int n_kv_heads, int head_dim, int page_size, int max_pages,
-                        double scale, const uint16_t *q, const uint16_t *k_pages, const uint16_t *v_pages,
+                        int window, double scale, const uint16_t *q, const uint16_t *k_pages, const uint16_t *v_pages,
                         const int32_t *page_table, const int32_t *seq_lens, double *out, double *lse)
 {
     int group = n_q_heads / n_kv_heads;
@@ -84,10 +89,11 @@ void oracle_verify_attn(int B, int R, int n_q_heads, int n_kv_heads, int head_di
         int b = (int)(item / ((long)n_q_heads * R));
         int g = h / group;
         int n_ctx = seq_lens[b] + j + 1;
+        int first = (window > 0 && n_ctx > window) ? n_ctx - window : 0;   /* oldest visible position */
         const uint16_t *qv = q + (size_t)item * head_dim;
         double *s = (double *)malloc(sizeof(double) * (size_t)n_ctx);
         double m = -INFINITY;
-        for (int i = 0; i < n_ctx; ++i) {
+        for (int i = first; i < n_ctx; ++i) {
             double acc = 0.0;
             for (int c = 0; c < head_dim; ++c)
                 acc += bf16_to_f64(qv[c]) *
@@ -96,10 +102,10 @@ void oracle_verify_attn(int B, int R, int n_q_heads, int n_kv_heads, int head_di
             if (s[i] > m) m = s[i];
         }
         double l = 0.0;
-        for (int i = 0; i < n_ctx; ++i) l += exp(s[i] - m);
+        for (int i = first; i < n_ctx; ++i) l += exp(s[i] - m);
         double *o = out + (size_t)item * head_dim;
         for (int c = 0; c < head_dim; ++c) o[c] = 0.0;
-        for (int i = 0; i < n_ctx; ++i) {
+        for (int i = first; i < n_ctx; ++i) {
             double w = exp(s[i] - m) / l;
             for (int c = 0; c < head_dim; ++c)
                 o[c] += w * bf16_to_f64(v_pages[kv_index(page_table, max_pages, page_size, n_kv_heads, head_dim, b, i, g, c)]);

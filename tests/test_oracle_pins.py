@@ -517,3 +517,53 @@ def test_flat_vocab_acceptance_rate_matches_gaussian_closed_form():
     exp_rate = np.minimum(p, q).sum(-1)
     assert abs(exp_rate.mean() - 2 * 0.5 * math.erfc(0.5 / math.sqrt(2))) < 0.05
     assert 1 <= int(res["accept_len"][0]) <= cfg.rows
+
+
+# ----------------------------------------------------------------------------- sliding-window attention
+
+def test_window_matches_library_softmax_with_band_mask():
+    rng = np.random.default_rng(31)
+    seq_lens, R, Hq, Hkv, d = [0, 5, 16, 37], 4, 4, 2, 8
+    w = make_paged(rng, seq_lens, R, Hq, Hkv, d)
+    oracle.kv_append(w["k_new"], w["v_new"], w["k_pages"], w["v_pages"], w["page_table"], w["seq_lens"])
+    q = from_bits(w["q"])
+    G = Hq // Hkv
+    for window in (1, 3, 7, 100):
+        out, lse = oracle.verify_attn(w["q"], w["k_pages"], w["v_pages"], w["page_table"], w["seq_lens"], window=window)
+        for b, L in enumerate(seq_lens):
+            Kl, Vl = logical_kv(w, b, L + R)
+            pos = np.arange(L + R)[None, :]
+            row_pos = (L + np.arange(R))[:, None]
+            hidden = (pos > row_pos) | (pos < row_pos - window + 1)
+            for h in range(Hq):
+                s = q[b, :, h, :] @ Kl[:, h // G, :].T / math.sqrt(d)
+                s = np.where(hidden, -np.inf, s)
+                pr = scipy.special.softmax(s, axis=-1)
+                np.testing.assert_allclose(out[b, :, h, :], pr @ Vl[:, h // G, :], rtol=0, atol=1e-12)
+                np.testing.assert_allclose(lse[b, :, h], scipy.special.logsumexp(s, axis=-1), rtol=0, atol=1e-12)
+
+
+def test_window_closed_forms():
+    """Window 1: every row returns its own value.  Zero keys: the mean of V over the last
+    `window` positions.  A window at least as long as the context is full attention."""
+    rng = np.random.default_rng(32)
+    L, R, d = 21, 5, 4
+    w = make_paged(rng, [L], R, 2, 2, d)
+    w["k_pages"][:] = 0
+    w["k_new"][:] = 0
+    vals = np.zeros(from_bits(w["v_pages"]).shape)
+    for pos in range(L):
+        vals[w["page_table"][0, pos // 16], :, pos % 16, :] = pos
+    w["v_pages"] = to_bits(vals)
+    w["v_new"] = to_bits(np.broadcast_to((L + np.arange(R))[None, :, None, None], (1, R, 2, d)).copy())
+    oracle.kv_append(w["k_new"], w["v_new"], w["k_pages"], w["v_pages"], w["page_table"], w["seq_lens"])
+    args = (w["q"], w["k_pages"], w["v_pages"], w["page_table"], w["seq_lens"])
+    out1, _ = oracle.verify_attn(*args, window=1)
+    out6, lse6 = oracle.verify_attn(*args, window=6)
+    full, lse_full = oracle.verify_attn(*args)
+    wide, lse_wide = oracle.verify_attn(*args, window=L + R)
+    for j in range(R):
+        np.testing.assert_allclose(out1[0, j], L + j, atol=1e-12)
+        np.testing.assert_allclose(out6[0, j], L + j - 2.5, atol=1e-12)        # mean of the last six positions
+        np.testing.assert_allclose(lse6[0, j], math.log(6), atol=1e-12)
+    assert np.array_equal(full, wide) and np.array_equal(lse_full, lse_wide)
