@@ -68,6 +68,7 @@ typedef struct massv_attn_desc {
     int64_t num_pages;           /* pages in the pool */
     float scale;                 /* score scale; 0 selects 1/sqrt(d) */
     int32_t kv_chunk;            /* tokens per split of the KV scan, multiple of 64, <= 4096; 0 = choose automatically */
+    int32_t window;              /* sliding-window attention: a row sees only its last `window` positions; 0 = full */
     uint32_t flags;              /* reserved, 0 */
 } massv_attn_desc;
 
@@ -97,6 +98,8 @@ size_t massv_verify_attn_workspace_size(const massv_attn_desc *desc);
  *      positions i = 0 .. L_b + j of KV head h / (Hq/Hkv): the whole committed
  *      prefix and the block rows up to and including j (causal inside the block).
  * Q and cached K are used as given (any positional encoding is already applied).
+ * With desc->window = w > 0 the sum runs over positions max(0, L_b + j - w + 1) .. L_b + j only
+ * (local attention layers; Sec. 4 of the paper notes Gemma3's interleaved sliding-window layers).
  *
  *   q                bf16 [B, R, Hq, d]
  *   k_new, v_new     bf16 [B, R, Hkv, d]

@@ -27,7 +27,7 @@ class AttnDesc(ctypes.Structure):
     _fields_ = [("batch", ctypes.c_int32), ("gamma", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
                 ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
                 ("max_pages_per_seq", ctypes.c_int32), ("num_pages", ctypes.c_int64), ("scale", ctypes.c_float),
-                ("kv_chunk", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+                ("kv_chunk", ctypes.c_int32), ("window", ctypes.c_int32), ("flags", ctypes.c_uint32)]
 
 
 class AcceptDesc(ctypes.Structure):
@@ -99,9 +99,9 @@ def massv_strerror(status: int) -> str:
 
 
 def attn_desc(batch, gamma, n_q_heads, n_kv_heads, head_dim, max_pages_per_seq, num_pages, scale=0.0, kv_chunk=0,
-              page_size=16) -> AttnDesc:
+              page_size=16, window=0) -> AttnDesc:
     return AttnDesc(batch, gamma, n_q_heads, n_kv_heads, head_dim, page_size, max_pages_per_seq, num_pages,
-                    float(scale), kv_chunk, 0)
+                    float(scale), kv_chunk, window, 0)
 
 
 def accept_desc(batch, gamma, hidden, vocab, temperature) -> AcceptDesc:

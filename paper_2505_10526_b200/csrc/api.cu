@@ -36,7 +36,7 @@ int auto_kv_chunk(const massv_attn_desc& d) {
 int check_attn_desc(const massv_attn_desc* d) {
     if (!d) return MASSV_ERR_INVALID_ARG;
     if (d->batch < 1 || d->n_q_heads < 1 || d->n_kv_heads < 1 || d->max_pages_per_seq < 1 || d->num_pages < 1 ||
-        d->gamma < 0 || d->scale < 0.f || d->kv_chunk < 0)
+        d->gamma < 0 || d->scale < 0.f || d->kv_chunk < 0 || d->window < 0)
         return MASSV_ERR_INVALID_ARG;
     if (d->gamma > kMaxRows - 1) return MASSV_ERR_UNSUPPORTED;
     if (d->page_size != kPageSize) return MASSV_ERR_UNSUPPORTED;
@@ -127,7 +127,7 @@ int massv_verify_attn(const massv_attn_desc* desc, const void* q, const void* k_
     p.B = desc->batch; p.R = desc->gamma + 1; p.Hq = desc->n_q_heads; p.Hkv = desc->n_kv_heads;
     p.d = desc->head_dim; p.max_pages = desc->max_pages_per_seq; p.num_pages = desc->num_pages;
     p.scale = desc->scale > 0.f ? desc->scale : 1.f / sqrtf((float)desc->head_dim);
-    p.kv_chunk = l.kv_chunk; p.max_chunks = l.max_chunks;
+    p.kv_chunk = l.kv_chunk; p.max_chunks = l.max_chunks; p.window = desc->window;
     p.q = static_cast<const __nv_bfloat16*>(q);
     p.k_new = static_cast<const __nv_bfloat16*>(k_new);
     p.v_new = static_cast<const __nv_bfloat16*>(v_new);

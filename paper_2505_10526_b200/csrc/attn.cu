@@ -91,11 +91,18 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
         return;
     }
     const int n_ctx = L + p.R;
-    const int c_begin = chunk * p.kv_chunk;
-    if (c_begin >= n_ctx) return;
-    const int c_end = min(n_ctx, c_begin + p.kv_chunk);
+    if (chunk * p.kv_chunk >= n_ctx) return;
+    // Sliding window: block row j (position L + j) sees positions L + j - window + 1 .. L + j, so
+    // nothing before row 0's lower bound is needed.  Chunks wholly before it retire, and the
+    // first needed chunk starts at the tile that holds the bound.
+    const int lo_min = p.window > 0 ? max(0, L - p.window + 1) : 0;
+    const int first_chunk = lo_min / p.kv_chunk;
+    if (chunk < first_chunk) return;
+    int c_begin = chunk * p.kv_chunk;
+    if (chunk == first_chunk) c_begin += ((lo_min - c_begin) / kTile) * kTile;
+    const int c_end = min(n_ctx, chunk * p.kv_chunk + p.kv_chunk);
     const int n_tiles = (c_end - c_begin + kTile - 1) / kTile;
-    const int n_chunks_b = (n_ctx + p.kv_chunk - 1) / p.kv_chunk;
+    const int n_chunks_b = (n_ctx + p.kv_chunk - 1) / p.kv_chunk - first_chunk;     // chunks that take part
     const int G = p.Hq / p.Hkv;
     const int rows = G * p.R;
 
@@ -246,7 +253,9 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
             }
 
             // ---- scale, causal mask, online softmax
-            const bool need_mask = tile_start + kTile > L + 1;   // some position in the tile is hidden from block row 0
+            // some position in the tile is hidden from some block row: ahead of row 0, or (with a
+            // window) older than the last row's lower bound
+            const bool need_mask = tile_start + kTile > L + 1 || (p.window > 0 && tile_start < n_ctx - p.window);
             float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
             for (int n = 0; n < NT / 8; ++n) {
@@ -255,7 +264,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_consta
                     float sv = sacc[n][e] * scale_log2;
                     if (need_mask) {
                         const int pos = tile_start + ts * NT + n * 8 + 2 * (lane & 3) + (e & 1);
-                        if (pos > L + (e < 2 ? j0 : j1)) sv = -INFINITY;
+                        const int row_pos = L + (e < 2 ? j0 : j1);
+                        if (pos > row_pos || (p.window > 0 && pos < row_pos - p.window + 1)) sv = -INFINITY;
                     }
                     sacc[n][e] = sv;
                     if (e < 2) mx0 = fmaxf(mx0, sv); else mx1 = fmaxf(mx1, sv);
@@ -376,11 +386,12 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const AttnParams p, i
     pdl_trigger();
     const int L = p.seq_lens[b];
     if (L < 0 || L + p.R > p.max_pages * kPageSize) return;
-    const int n_chunks = (L + p.R + p.kv_chunk - 1) / p.kv_chunk;
+    const int first_chunk = (p.window > 0 ? max(0, L - p.window + 1) : 0) / p.kv_chunk;   // as in the split kernel
+    const int n_chunks = (L + p.R + p.kv_chunk - 1) / p.kv_chunk - first_chunk;
     if (n_chunks <= 1) return;
     __shared__ float s_w[kCombineMaxChunks];    // first the chunk maxima, then the merge weights
     __shared__ float s_l[kCombineMaxChunks];
-    const size_t item0 = ((size_t)b * p.Hkv + g) * p.max_chunks;
+    const size_t item0 = ((size_t)b * p.Hkv + g) * p.max_chunks + first_chunk;
     for (int c = threadIdx.x; c < n_chunks; c += blockDim.x) {
         const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((item0 + c) * rows_pad + r) * 2);
         s_w[c] = ml.x;

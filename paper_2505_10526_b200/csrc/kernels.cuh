@@ -10,6 +10,7 @@ struct AttnParams {
     int B, R, Hq, Hkv, d, max_pages;
     int64_t num_pages;
     float scale;
+    int window;        // sliding window length, 0 = full attention
     int kv_chunk;      // tokens per split
     int max_chunks;    // splits launched per (sequence, kv head)
     const __nv_bfloat16 *q, *k_new, *v_new;

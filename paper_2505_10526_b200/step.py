@@ -17,13 +17,13 @@ STEP_INPUTS = ("q", "k_new", "v_new", "hidden", "draft_tokens", "draft_probs", "
 
 class VerifyStep:
     def __init__(self, batch, gamma, n_q_heads, n_kv_heads, head_dim, hidden, vocab, temperature,
-                 max_pages_per_seq, num_pages, device="cuda", kv_chunk=0, scale=0.0,
+                 max_pages_per_seq, num_pages, device="cuda", kv_chunk=0, scale=0.0, window=0,
                  want_logits=False, want_probs=False, want_attn_f32=False):
         self.device = torch.device(device)
         self.B, self.gamma, self.R = batch, gamma, gamma + 1
         self.T = float(temperature)
         self.adesc = mv.attn_desc(batch, gamma, n_q_heads, n_kv_heads, head_dim, max_pages_per_seq, num_pages,
-                                  scale=scale, kv_chunk=kv_chunk)
+                                  scale=scale, kv_chunk=kv_chunk, window=window)
         self.cdesc = mv.accept_desc(batch, gamma, hidden, vocab, temperature)
         dev = self.device
         self.attn_ws = mv.alloc_workspace(mv.massv_verify_attn_workspace_size(self.adesc), dev)
@@ -44,7 +44,7 @@ class VerifyStep:
     def for_workload(cls, cfg, w, **kw):
         return cls(cfg.batch, cfg.gamma, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.hidden, cfg.vocab,
                    cfg.temperature, w["page_table"].shape[1], w["k_pages"].shape[0],
-                   device=w["k_pages"].device, **kw)
+                   device=w["k_pages"].device, **{"window": getattr(cfg, "window", 0), **kw})
 
     # -- the three calls -------------------------------------------------------------
     def attn(self, w):

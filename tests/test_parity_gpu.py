@@ -34,13 +34,13 @@ def _report(entry):
     print(entry)
 
 
-def run_case(name, subset=None, check_determinism=True, cfg=None, **step_kw):
+def run_case(name, subset=None, check_determinism=True, cfg=None, window=0, **step_kw):
     from paper_2505_10526_b200 import VerifyStep
     cfg = cfg or get_config(name)
     w = generate(cfg, device="cuda")
     pools_before = (w["k_pages"].clone(), w["v_pages"].clone())
     seq_before = w["seq_lens"].clone()
-    step = VerifyStep.for_workload(cfg, w, want_logits=True, want_probs=True, want_attn_f32=True, **step_kw)
+    step = VerifyStep.for_workload(cfg, w, want_logits=True, want_probs=True, want_attn_f32=True, window=window, **step_kw)
     step.run(w, commit=True)
     torch.cuda.synchronize()
     assert int(step.dev_status.item()) == 0
@@ -50,7 +50,7 @@ def run_case(name, subset=None, check_determinism=True, cfg=None, **step_kw):
     w_ref = dict(w)
     w_ref["k_pages"], w_ref["v_pages"] = pools_before
     w_ref["seq_lens"] = seq_before
-    ref = oracle.verify_step(sub_workload(w_ref, idx), cfg.temperature)
+    ref = oracle.verify_step(sub_workload(w_ref, idx), cfg.temperature, window=window)
     R, V = cfg.rows, cfg.vocab
     sel = torch.as_tensor(idx, device="cuda")
 
@@ -217,3 +217,16 @@ def test_odd_shapes_and_forced_splits(spec, kv_chunk):
     from workloads import VerifyConfig
     cfg = VerifyConfig(image_tokens=0.25, draft_noise_std=0.7, seed=40 + len(spec["name"]), **spec)
     run_case(None, cfg=cfg, kv_chunk=kv_chunk)
+
+
+@pytest.mark.parametrize("name,window,kv_chunk,subset", [
+    ("tiny_ragged_t1", 1, 0, None), ("tiny_ragged_t1", 5, 64, None), ("tiny_ragged_t0", 40, 64, None),
+    ("tiny_t1", 100, 64, None), ("tiny_t1", 1000, 0, None),
+    ("qwen7b_b16_t1", 512, 0, None), ("qwen7b_b16_t1", 1500, 256, None),
+    ("gemma12b_b32_t1", 1024, 0, [0, 7, 19, 31]),
+])
+def test_sliding_window_attention(name, window, kv_chunk, subset):
+    """Local-attention variant: each block row sees only its last `window` positions.  Windows
+    shorter than, comparable to and longer than the context, with automatic and forced chunking
+    (whole chunks before the window are skipped; the first needed chunk starts mid-way)."""
+    run_case(name, subset=subset, check_determinism=False, window=window, kv_chunk=kv_chunk)

@@ -29,6 +29,7 @@ class VerifyConfig:
     draft_noise_std: float     # std of the Gaussian noise added to target logits to form the drafter
     seed: int
     hidden_std: float = 1.0    # std of the hidden states (4.0 gives peaked distributions)
+    window: int = 0            # sliding-window attention length (0 = full attention)
     page_size: int = 16
 
     @property
@@ -87,6 +88,8 @@ _add(VerifyConfig("tiny_ragged_t0", 5, 7, **_TINY, temperature=0.0, ctx_lo=0, ct
 _add(replace(CONFIGS["qwen7b_b16_t1"], name="qwen7b_b16_t1_peaked", hidden_std=5.0, seed=13))
 
 
+# A local-attention layer of the Gemma3-shaped target (sliding window of 1024 positions).
+_add(replace(CONFIGS["gemma12b_b32_t1"], name="gemma12b_b32_t1_local", window=1024))
 # Reduced-batch copies of the long-context points, small enough for multi-pass profiler captures.
 for _g in (5, 7):
     _add(replace(CONFIGS[f"qwen7b_long_g{_g}_t0"], name=f"qwen7b_long_b16_g{_g}_t0", batch=16))

@@ -37,7 +37,8 @@ def _randn_bf16(shape, std, gen, device, chunk_rows=16384):
 def kv_bytes(cfg: VerifyConfig, seq_lens) -> int:
     """Bytes of K and V that one verify step must read: every cached position
     plus the gamma+1 appended ones, once each, for every KV head."""
-    tot = int(sum(int(l) + cfg.rows for l in seq_lens))
+    w = getattr(cfg, "window", 0)
+    tot = int(sum(min(int(l) + cfg.rows, w + cfg.rows - 1) if w > 0 else int(l) + cfg.rows for l in seq_lens))
     return tot * cfg.n_kv_heads * cfg.head_dim * 2 * 2
 
 
