@@ -24,7 +24,9 @@ int auto_kv_chunk(const massv_attn_desc& d) {
     // Large problems: about five waves of CTAs (two per SM), but chunks of at least 768 tokens
     // so that the partial results written per chunk stay a few percent of the K/V read.
     // Small problems (too few CTAs that way): split down to 64 tokens to fill the machine.
-    const double th = (double)d.batch * d.max_pages_per_seq * kPageSize * d.n_kv_heads;
+    long per_seq_tokens = (long)d.max_pages_per_seq * kPageSize;
+    if (d.window > 0 && d.window + 64 < per_seq_tokens) per_seq_tokens = d.window + 64;   // only the window is read
+    const double th = (double)d.batch * per_seq_tokens * d.n_kv_heads;
     long chunk = ((long)ceil(th / 1480.0) + 63) / 64 * 64;
     if (chunk < 768) chunk = 768;
     if (th / (double)chunk < 128.0) chunk = ((long)ceil(th / 128.0) + 63) / 64 * 64;
