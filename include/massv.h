@@ -201,6 +201,27 @@ int massv_accept_static(const massv_accept_desc *desc, const void *hidden, const
                         int32_t *out_tokens, int32_t *accept_len, float *logits_out, float *probs_out,
                         int32_t *dev_status, massv_stream_t stream);
 
+/* Bytes of scratch massv_tvd needs (0 on a bad descriptor, gamma == 0 or T == 0). */
+size_t massv_tvd_workspace_size(const massv_accept_desc *desc);
+
+/*
+ * Distribution-alignment diagnostic of the paper (Eq. 6): for every drafted
+ * position (b, j), the total variation distance between the target distribution
+ * p_j = softmax(z_j / T) and the draft distribution q_j,
+ *     tvd_out[b,j] = 1/2 * sum_v |p_j(v) - q_j(v)|   in [0, 1],
+ * and optionally accept_prob_out[b,j] = sum_v min(p_j(v), q_j(v)) = 1 - TVD, the
+ * probability that the rejection test of massv_accept accepts a draft token
+ * drawn from q_j.
+ *   logits        fp32 [B, R, V]   (the logits_out of massv_accept; rows 0..gamma-1 are used)
+ *   draft_probs   fp32 [B, gamma, V]
+ *   tvd_out       fp32 [B, gamma];  accept_prob_out  optional fp32 [B, gamma]
+ * Needs T > 0 and gamma >= 1.  Reads every drafted row once (B*gamma*V*8 bytes),
+ * twice for the logits; sums run in fp64 in a fixed order.
+ */
+int massv_tvd(const massv_accept_desc *desc, const float *logits, const float *draft_probs,
+              float *tvd_out, float *accept_prob_out,
+              void *workspace, size_t workspace_bytes, int32_t *dev_status, massv_stream_t stream);
+
 /*
  * Commit or roll back the speculative block (Sec. 2.1: accepted tokens are
  * added to the output and the next iteration starts from them).

@@ -54,6 +54,10 @@ def _load():
     lib.massv_accept_static.restype = ctypes.c_int
     lib.massv_accept_static.argtypes = [ctypes.POINTER(AcceptDesc), vp, vp, i32p, f32p, f32p, f32p, i32p, i32p, f32p, f32p,
                                         i32p, vp]
+    lib.massv_tvd_workspace_size.restype = ctypes.c_size_t
+    lib.massv_tvd_workspace_size.argtypes = [ctypes.POINTER(AcceptDesc)]
+    lib.massv_tvd.restype = ctypes.c_int
+    lib.massv_tvd.argtypes = [ctypes.POINTER(AcceptDesc), f32p, f32p, f32p, f32p, vp, ctypes.c_size_t, i32p, vp]
     lib.massv_kv_commit.restype = ctypes.c_int
     lib.massv_kv_commit.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, vp]
     lib.massv_strerror.restype = ctypes.c_char_p
@@ -157,6 +161,19 @@ def massv_accept_static(desc, hidden, lm_head, draft_tokens, draft_probs, u_acce
                                   _ptr(probs_out, f32), _ptr(dev_status, i32), _stream())
     if rc != 0:
         raise MassvError(rc, "massv_accept_static")
+
+
+def massv_tvd_workspace_size(desc: AcceptDesc) -> int:
+    return int(_lib.massv_tvd_workspace_size(ctypes.byref(desc)))
+
+
+def massv_tvd(desc, logits, draft_probs, tvd_out, accept_prob_out=None, workspace=None, dev_status=None) -> None:
+    f32 = torch.float32
+    rc = _lib.massv_tvd(ctypes.byref(desc), _ptr(logits, f32), _ptr(draft_probs, f32), _ptr(tvd_out, f32),
+                        _ptr(accept_prob_out, f32), _ptr(workspace), workspace.numel() if workspace is not None else 0,
+                        _ptr(dev_status, torch.int32), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_tvd")
 
 
 def massv_kv_commit(batch, gamma, accept_len, seq_lens, dev_status=None) -> None:

@@ -199,6 +199,35 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
     return launch_accept(a, s) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
+size_t massv_tvd_workspace_size(const massv_accept_desc* desc) {
+    if (check_accept_desc(desc) != MASSV_OK || desc->gamma < 1 || !(desc->temperature > 0.f)) return 0;
+    const size_t rows = (size_t)desc->batch * desc->gamma;
+    return align_up(rows * kTvdSlices * sizeof(float), kAlign) + 3 * align_up(rows * kTvdSlices * sizeof(double), kAlign);
+}
+
+int massv_tvd(const massv_accept_desc* desc, const float* logits, const float* draft_probs, float* tvd_out,
+              float* accept_prob_out, void* workspace, size_t workspace_bytes, int32_t* dev_status, massv_stream_t stream) {
+    (void)dev_status;
+    const int rc = check_accept_desc(desc);
+    if (rc != MASSV_OK) return rc;
+    if (desc->gamma < 1 || !(desc->temperature > 0.f)) return MASSV_ERR_INVALID_ARG;
+    if (!logits || !draft_probs || !tvd_out) return MASSV_ERR_INVALID_ARG;
+    const size_t need = massv_tvd_workspace_size(desc);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0 || workspace_bytes < need) return MASSV_ERR_WORKSPACE;
+    const size_t rows = (size_t)desc->batch * desc->gamma;
+    char* ws = static_cast<char*>(workspace);
+    TvdParams t;
+    t.B = desc->batch; t.gamma = desc->gamma; t.V = desc->vocab; t.inv_T = 1.f / desc->temperature;
+    t.slice_len = (desc->vocab + kTvdSlices - 1) / kTvdSlices;
+    t.logits = logits; t.draft_probs = draft_probs; t.tvd_out = tvd_out; t.accept_prob_out = accept_prob_out;
+    t.slice_max = reinterpret_cast<float*>(ws);
+    const size_t off = align_up(rows * kTvdSlices * sizeof(float), kAlign), step = align_up(rows * kTvdSlices * sizeof(double), kAlign);
+    t.slice_sum = reinterpret_cast<double*>(ws + off);
+    t.slice_abs = reinterpret_cast<double*>(ws + off + step);
+    t.slice_min = reinterpret_cast<double*>(ws + off + 2 * step);
+    return launch_tvd(t, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
 int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
                     massv_stream_t stream) {
     if (batch < 1 || gamma < 0 || !seq_lens) return MASSV_ERR_INVALID_ARG;

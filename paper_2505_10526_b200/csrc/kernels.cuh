@@ -61,6 +61,19 @@ struct AcceptParams {
 };
 cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream);
 
+// ---------------------------------------------------------------- TVD diagnostic
+constexpr int kTvdSlices = 16;      // vocabulary slices per row
+struct TvdParams {
+    int B, gamma, V;
+    float inv_T;
+    int slice_len;                  // entries per slice
+    const float *logits, *draft_probs;
+    float *tvd_out, *accept_prob_out;
+    float* slice_max;               // [B*gamma, kTvdSlices]
+    double *slice_sum, *slice_abs, *slice_min;
+};
+cudaError_t launch_tvd(const TvdParams& p, cudaStream_t stream);
+
 cudaError_t launch_kv_commit(int B, int gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
                              cudaStream_t stream);
 

@@ -1,0 +1,123 @@
+// Total variation distance between the target's and the drafter's token
+// distributions for every drafted position (paper Eq. 6):
+//     TVD(p_j, q_j) = 1/2 * sum_v |p_j(v) - q_j(v)|,      p_j = softmax(z_j / T)
+// and the acceptance probability of the rejection test, sum_v min(p_j(v), q_j(v)) = 1 - TVD.
+// Three small kernels over fixed vocabulary slices, every reduction in a fixed order:
+//   tvd_stats_kernel   per (row, slice): max logit and sum of exponentials;
+//   tvd_sum_kernel     per (row, slice): merge the row's slice statistics, then sum |p-q| and min(p,q);
+//   tvd_final_kernel   per row: add the slices in order.
+#include "kernels.cuh"
+
+namespace massv {
+
+namespace {
+
+constexpr int kThreadsTvd = 256;
+
+// Sum over the block in a fixed tree; valid in thread 0.
+__device__ __forceinline__ double block_sum(double x, double* sh) {
+    sh[threadIdx.x] = x;
+    __syncthreads();
+    for (int w = kThreadsTvd / 2; w > 0; w >>= 1) {
+        if (threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+        __syncthreads();
+    }
+    const double r = sh[0];
+    __syncthreads();
+    return r;
+}
+__device__ __forceinline__ float block_max(float x, float* sh) {
+    sh[threadIdx.x] = x;
+    __syncthreads();
+    for (int w = kThreadsTvd / 2; w > 0; w >>= 1) {
+        if (threadIdx.x < w) sh[threadIdx.x] = fmaxf(sh[threadIdx.x], sh[threadIdx.x + w]);
+        __syncthreads();
+    }
+    const float r = sh[0];
+    __syncthreads();
+    return r;
+}
+
+// Row r of the drafted positions = (sequence b, draft j): logits row b*(gamma+1)+j, q row b*gamma+j.
+__device__ __forceinline__ const float* logits_row(const TvdParams& p, int row) {
+    const int b = row / p.gamma, j = row % p.gamma;
+    return p.logits + (size_t)(b * (p.gamma + 1) + j) * p.V;
+}
+
+__global__ void __launch_bounds__(kThreadsTvd) tvd_stats_kernel(TvdParams p) {
+    __shared__ float shf[kThreadsTvd];
+    __shared__ double shd[kThreadsTvd];
+    pdl_wait();
+    pdl_trigger();
+    const int slice = blockIdx.x, row = blockIdx.y;
+    const int v0 = slice * p.slice_len, v1 = min(p.V, v0 + p.slice_len);
+    const float* z = logits_row(p, row);
+    float m = -INFINITY;
+    for (int v = v0 + threadIdx.x; v < v1; v += kThreadsTvd) m = fmaxf(m, z[v]);
+    m = block_max(m, shf);
+    double s = 0.0;
+    if (m > -INFINITY)
+        for (int v = v0 + threadIdx.x; v < v1; v += kThreadsTvd) s += (double)expf((z[v] - m) * p.inv_T);
+    s = block_sum(s, shd);
+    if (threadIdx.x == 0) {
+        p.slice_max[row * kTvdSlices + slice] = m;
+        p.slice_sum[row * kTvdSlices + slice] = s;
+    }
+}
+
+__global__ void __launch_bounds__(kThreadsTvd) tvd_sum_kernel(TvdParams p) {
+    __shared__ double shd[kThreadsTvd];
+    pdl_wait();
+    pdl_trigger();
+    const int slice = blockIdx.x, row = blockIdx.y;
+    float M = -INFINITY;
+    for (int s = 0; s < kTvdSlices; ++s) M = fmaxf(M, p.slice_max[row * kTvdSlices + s]);
+    double S = 0.0;
+    for (int s = 0; s < kTvdSlices; ++s) {
+        const float ms = p.slice_max[row * kTvdSlices + s];
+        if (ms > -INFINITY) S += p.slice_sum[row * kTvdSlices + s] * (double)expf((ms - M) * p.inv_T);
+    }
+    const float inv_sum = (float)(1.0 / S);
+    const int v0 = slice * p.slice_len, v1 = min(p.V, v0 + p.slice_len);
+    const float* z = logits_row(p, row);
+    const float* q = p.draft_probs + (size_t)row * p.V;
+    double a = 0.0, mn = 0.0;
+    for (int v = v0 + threadIdx.x; v < v1; v += kThreadsTvd) {
+        const float pv = expf((z[v] - M) * p.inv_T) * inv_sum;
+        const float qv = q[v];
+        a += (double)fabsf(pv - qv);
+        mn += (double)fminf(pv, qv);
+    }
+    a = block_sum(a, shd);
+    mn = block_sum(mn, shd);
+    if (threadIdx.x == 0) {
+        p.slice_abs[row * kTvdSlices + slice] = a;
+        p.slice_min[row * kTvdSlices + slice] = mn;
+    }
+}
+
+__global__ void tvd_final_kernel(TvdParams p) {
+    pdl_wait();
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= p.B * p.gamma) return;
+    double a = 0.0, mn = 0.0;
+    for (int s = 0; s < kTvdSlices; ++s) { a += p.slice_abs[row * kTvdSlices + s]; mn += p.slice_min[row * kTvdSlices + s]; }
+    p.tvd_out[row] = (float)(0.5 * a);
+    if (p.accept_prob_out) p.accept_prob_out[row] = (float)mn;
+}
+
+}  // namespace
+
+cudaError_t launch_tvd(const TvdParams& p, cudaStream_t stream) {
+    const int rows = p.B * p.gamma;
+    cudaError_t e = launch_pdl(tvd_stats_kernel, dim3(kTvdSlices, rows), dim3(kThreadsTvd), 0, stream, p);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(tvd_sum_kernel, dim3(kTvdSlices, rows), dim3(kThreadsTvd), 0, stream, p);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(tvd_final_kernel, dim3((rows + 127) / 128), dim3(128), 0, stream, p);
+    if (e != cudaSuccess) return e;
+    count_launches(3);
+    return cudaGetLastError();
+}
+
+}  // namespace massv

@@ -567,3 +567,12 @@ def test_window_closed_forms():
         np.testing.assert_allclose(out6[0, j], L + j - 2.5, atol=1e-12)        # mean of the last six positions
         np.testing.assert_allclose(lse6[0, j], math.log(6), atol=1e-12)
     assert np.array_equal(full, wide) and np.array_equal(lse_full, lse_wide)
+
+
+def test_tvd_hand_values():
+    """Eq. 6 on values worked by hand: identical -> 0, disjoint -> 1, and a three-token case."""
+    a = np.array([0.5, 0.3, 0.2]); b = np.array([0.2, 0.5, 0.3])
+    assert abs(oracle.tvd(a, b) - 0.3) < 1e-15            # (0.3 + 0.2 + 0.1) / 2
+    assert oracle.tvd(a, a.copy()) == 0.0
+    assert abs(oracle.tvd(np.array([1.0, 0.0, 0.0]), np.array([0.0, 0.25, 0.75])) - 1.0) < 1e-15
+    assert abs(oracle.tvd(a, b) - oracle.tvd(b, a)) < 1e-18

@@ -230,3 +230,34 @@ def test_sliding_window_attention(name, window, kv_chunk, subset):
     shorter than, comparable to and longer than the context, with automatic and forced chunking
     (whole chunks before the window are skipped; the first needed chunk starts mid-way)."""
     run_case(name, subset=subset, check_determinism=False, window=window, kv_chunk=kv_chunk)
+
+
+@pytest.mark.parametrize("name,subset", [("tiny_ragged_t1", None), ("tiny_peaked_t1", None), ("qwen7b_b16_t1", [0, 5, 15])])
+def test_tvd_diagnostic_matches_oracle(name, subset):
+    """massv_tvd (Eq. 6) against the oracle's TVD of (softmax of oracle logits, q), row by row;
+    1 - TVD must equal the acceptance probability output.  Tolerance 1e-4 absolute, the
+    tolerance of the probabilities it is a sum of differences of."""
+    import paper_2505_10526_b200 as mv
+    cfg = get_config(name)
+    w = generate(cfg, device="cuda", with_attention=False)
+    B, R, g, V = cfg.batch, cfg.rows, cfg.gamma, cfg.vocab
+    desc = mv.accept_desc(B, g, cfg.hidden, V, cfg.temperature)
+    ws = mv.alloc_workspace(mv.massv_accept_workspace_size(desc), "cuda")
+    toks = torch.zeros((B, R), dtype=torch.int32, device="cuda"); lens = torch.zeros((B,), dtype=torch.int32, device="cuda")
+    logits = torch.zeros((B, R, V), dtype=torch.float32, device="cuda")
+    mv.massv_accept(desc, w["hidden"], w["lm_head"], w["draft_tokens"], w["draft_probs"], w["u_accept"], w["u_sample"],
+                    toks, lens, logits, None, ws, None)
+    tvd = torch.zeros((B, g), dtype=torch.float32, device="cuda"); acc = torch.zeros_like(tvd)
+    ws2 = mv.alloc_workspace(mv.massv_tvd_workspace_size(desc), "cuda")
+    mv.massv_tvd(desc, logits, w["draft_probs"], tvd, acc, ws2, None)
+    torch.cuda.synchronize()
+    idx = list(range(B)) if subset is None else subset
+    hid = oracle.bf16_bits(w["hidden"])[idx].reshape(len(idx) * R, cfg.hidden)
+    p = oracle.softmax(oracle.logits(hid, oracle.bf16_bits(w["lm_head"])), cfg.temperature).reshape(len(idx), R, V)
+    q = w["draft_probs"].double().cpu().numpy()[idx]
+    for i, b in enumerate(idx):
+        for j in range(g):
+            ref = oracle.tvd(np.ascontiguousarray(p[i, j]), np.ascontiguousarray(q[i, j]))
+            assert abs(float(tvd[b, j]) - ref) < 1e-4, (b, j, float(tvd[b, j]), ref)
+            assert abs(float(acc[b, j]) - (1.0 - ref)) < 1e-4
+            assert 0.0 <= float(tvd[b, j]) <= 1.0 + 1e-6
