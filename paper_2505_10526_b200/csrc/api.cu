@@ -218,7 +218,7 @@ int massv_tvd(const massv_accept_desc* desc, const float* logits, const float* d
     char* ws = static_cast<char*>(workspace);
     TvdParams t;
     t.B = desc->batch; t.gamma = desc->gamma; t.V = desc->vocab; t.inv_T = 1.f / desc->temperature;
-    t.slice_len = (desc->vocab + kTvdSlices - 1) / kTvdSlices;
+    t.slice_len = ((desc->vocab + kTvdSlices - 1) / kTvdSlices + 3) / 4 * 4;      // 16-byte aligned slices (V % 8 == 0)
     t.logits = logits; t.draft_probs = draft_probs; t.tvd_out = tvd_out; t.accept_prob_out = accept_prob_out;
     t.slice_max = reinterpret_cast<float*>(ws);
     const size_t off = align_up(rows * kTvdSlices * sizeof(float), kAlign), step = align_up(rows * kTvdSlices * sizeof(double), kAlign);

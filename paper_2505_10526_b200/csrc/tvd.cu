@@ -52,12 +52,21 @@ __global__ void __launch_bounds__(kThreadsTvd) tvd_stats_kernel(TvdParams p) {
     const int slice = blockIdx.x, row = blockIdx.y;
     const int v0 = slice * p.slice_len, v1 = min(p.V, v0 + p.slice_len);
     const float* z = logits_row(p, row);
-    float m = -INFINITY;
-    for (int v = v0 + threadIdx.x; v < v1; v += kThreadsTvd) m = fmaxf(m, z[v]);
-    m = block_max(m, shf);
-    double s = 0.0;
-    if (m > -INFINITY)
-        for (int v = v0 + threadIdx.x; v < v1; v += kThreadsTvd) s += (double)expf((z[v] - m) * p.inv_T);
+    // one pass: every thread keeps a running (max, sum) over 16-byte loads, then the block merges
+    float tm = -INFINITY, ts = 0.f;
+    for (int v = v0 + 4 * threadIdx.x; v < v1; v += 4 * kThreadsTvd) {      // slices start at multiples of 4
+        const float4 x = *reinterpret_cast<const float4*>(z + v);
+        const float e[4] = {x.x, x.y, x.z, x.w};
+        float cm = tm;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) if (v + i < v1) cm = fmaxf(cm, e[i]);
+        float cs = tm == -INFINITY ? 0.f : ts * expf((tm - cm) * p.inv_T);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) if (v + i < v1) cs += expf((e[i] - cm) * p.inv_T);
+        tm = cm; ts = cs;
+    }
+    const float m = block_max(tm, shf);
+    double s = (tm == -INFINITY) ? 0.0 : (double)ts * (double)expf((tm - m) * p.inv_T);
     s = block_sum(s, shd);
     if (threadIdx.x == 0) {
         p.slice_max[row * kTvdSlices + slice] = m;
@@ -82,11 +91,21 @@ __global__ void __launch_bounds__(kThreadsTvd) tvd_sum_kernel(TvdParams p) {
     const float* z = logits_row(p, row);
     const float* q = p.draft_probs + (size_t)row * p.V;
     double a = 0.0, mn = 0.0;
-    for (int v = v0 + threadIdx.x; v < v1; v += kThreadsTvd) {
-        const float pv = expf((z[v] - M) * p.inv_T) * inv_sum;
-        const float qv = q[v];
-        a += (double)fabsf(pv - qv);
-        mn += (double)fminf(pv, qv);
+    for (int v = v0 + 4 * threadIdx.x; v < v1; v += 4 * kThreadsTvd) {
+        const float4 x = *reinterpret_cast<const float4*>(z + v);
+        const float4 y = __ldg(reinterpret_cast<const float4*>(q + v));
+        const float e[4] = {x.x, x.y, x.z, x.w}, f[4] = {y.x, y.y, y.z, y.w};
+        float fa = 0.f, fm = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (v + i < v1) {
+                const float pv = expf((e[i] - M) * p.inv_T) * inv_sum;
+                fa += fabsf(pv - f[i]);
+                fm += fminf(pv, f[i]);
+            }
+        }
+        a += (double)fa;
+        mn += (double)fm;
     }
     a = block_sum(a, shd);
     mn = block_sum(mn, shd);
