@@ -261,3 +261,29 @@ def test_tvd_diagnostic_matches_oracle(name, subset):
             assert abs(float(tvd[b, j]) - ref) < 1e-4, (b, j, float(tvd[b, j]), ref)
             assert abs(float(acc[b, j]) - (1.0 - ref)) < 1e-4
             assert 0.0 <= float(tvd[b, j]) <= 1.0 + 1e-6
+
+
+def test_gamma_zero_sampling_is_the_draft_side_step():
+    """With no drafts and T > 0 the call is one ordinary sampling step: the token is the
+    inverse-CDF draw from softmax(z / T) with the caller's uniform, and probs_out is that
+    distribution - which is exactly what a drafter must hand to the next verify step."""
+    from dataclasses import replace
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = replace(get_config("tiny_peaked_t1"), gamma=0, name="draft_step", batch=9, temperature=0.8)
+    w = generate(cfg, device="cuda")
+    step = VerifyStep.for_workload(cfg, w, want_logits=True, want_probs=True)
+    ref = oracle.verify_step({k: v.clone() for k, v in w.items()}, cfg.temperature)
+    step.run(w)
+    torch.cuda.synchronize()
+    st = compare_accept(ref, step.out_tokens.cpu().numpy(), step.accept_len.cpu().numpy(), 0)
+    assert st["hard"] == 0 and np.all(step.accept_len.cpu().numpy() == 1)
+    p = step.probs.cpu().double().numpy().reshape(cfg.batch, cfg.vocab)
+    assert np.abs(p - ref["probs"]).max() < TOL_PROB
+    np.testing.assert_allclose(p.sum(-1), 1.0, atol=1e-4)
+    # every drawn token has positive probability and lies where the uniform points in the CDF
+    toks = step.out_tokens.cpu().numpy()[:, 0]
+    u = w["u_sample"].cpu().numpy()[:, 0]
+    cdf = np.cumsum(ref["probs"], axis=-1)
+    for b in range(cfg.batch):
+        if ref["margin_sample"][b] >= 1e-3:
+            assert toks[b] == int(np.searchsorted(cdf[b], u[b] * cdf[b, -1], side="right"))
