@@ -168,6 +168,8 @@ def main():
     ap.add_argument("--config", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="massv", choices=["massv", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--attn-kernel", type=int, default=0, choices=[0, 1, 2],
+                    help="attention split kernel: 0 = chosen by shape, 1 = warp-level MMA, 2 = tcgen05")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -197,7 +199,7 @@ def main():
 
     cfg = get_config(args.config)
     w = generate(cfg, device=dev)
-    step = mv.VerifyStep.for_workload(cfg, w)
+    step = mv.VerifyStep.for_workload(cfg, w, attn_kernel=args.attn_kernel)
     seq0 = w["seq_lens"].clone()
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
@@ -308,6 +310,7 @@ def main():
         "config": {"workload": cfg.name, "batch": cfg.batch, "gamma": cfg.gamma, "temperature": cfg.temperature,
                    "n_q_heads": cfg.n_q_heads, "n_kv_heads": cfg.n_kv_heads, "head_dim": cfg.head_dim,
                    "hidden": cfg.hidden, "vocab": cfg.vocab, "mean_context": float(seq0.float().mean()),
+                   "attn_kernel": {0: "by shape", 1: "warp_mma", 2: "tcgen05"}[args.attn_kernel],
                    "l2": f"flushed between timed steps by a {L2_FLUSH_BYTES >> 20} MiB write; LM-head weights alone exceed L2",
                    "parallelism": f"replicas x{world}"},
         "breakdown_ms": {"verify_attn": t_attn, "accept": t_accept, "kv_commit": t_commit,

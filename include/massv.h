@@ -69,8 +69,15 @@ typedef struct massv_attn_desc {
     float scale;                 /* score scale; 0 selects 1/sqrt(d) */
     int32_t kv_chunk;            /* tokens per split of the KV scan, multiple of 64, <= 4096; 0 = choose automatically */
     int32_t window;              /* sliding-window attention: a row sees only its last `window` positions; 0 = full */
-    uint32_t flags;              /* reserved, 0 */
+    uint32_t flags;              /* kernel choice, one of MASSV_ATTN_KERNEL_*; 0 = by shape */
 } massv_attn_desc;
+
+/* massv_attn_desc.flags.  Both kernels compute the same thing to the same tolerance; the choice
+ * only matters for speed (the library picks by the number of query rows per KV head) and is
+ * exposed so that either kernel can be checked on any shape. */
+#define MASSV_ATTN_KERNEL_AUTO 0u
+#define MASSV_ATTN_KERNEL_WARP_MMA 1u   /* warp-level tensor-core MMAs, operands through registers */
+#define MASSV_ATTN_KERNEL_TCGEN05 2u    /* tcgen05 MMAs with accumulators in tensor memory */
 
 /* Geometry of the acceptance call. */
 typedef struct massv_accept_desc {

@@ -102,10 +102,14 @@ def massv_strerror(status: int) -> str:
     return _strerror(status)
 
 
+# massv_attn_desc.flags: which split kernel runs (include/massv.h)
+ATTN_KERNEL_AUTO, ATTN_KERNEL_WARP_MMA, ATTN_KERNEL_TCGEN05 = 0, 1, 2
+
+
 def attn_desc(batch, gamma, n_q_heads, n_kv_heads, head_dim, max_pages_per_seq, num_pages, scale=0.0, kv_chunk=0,
-              page_size=16, window=0) -> AttnDesc:
+              page_size=16, window=0, kernel=ATTN_KERNEL_AUTO) -> AttnDesc:
     return AttnDesc(batch, gamma, n_q_heads, n_kv_heads, head_dim, page_size, max_pages_per_seq, num_pages,
-                    float(scale), kv_chunk, window, 0)
+                    float(scale), kv_chunk, window, int(kernel))
 
 
 def accept_desc(batch, gamma, hidden, vocab, temperature) -> AcceptDesc:

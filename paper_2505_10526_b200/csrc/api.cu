@@ -46,7 +46,7 @@ int check_attn_desc(const massv_attn_desc* d) {
     if (d->n_q_heads % d->n_kv_heads != 0) return MASSV_ERR_UNSUPPORTED;
     if ((d->n_q_heads / d->n_kv_heads) * (d->gamma + 1) > 64) return MASSV_ERR_UNSUPPORTED;
     if (d->kv_chunk % 64 != 0 || d->kv_chunk > 4096) return MASSV_ERR_UNSUPPORTED;
-    if (d->flags != 0) return MASSV_ERR_UNSUPPORTED;
+    if (d->flags > MASSV_ATTN_KERNEL_TCGEN05) return MASSV_ERR_UNSUPPORTED;
     return MASSV_OK;
 }
 
@@ -141,6 +141,7 @@ int massv_verify_attn(const massv_attn_desc* desc, const void* q, const void* k_
     p.part_o = reinterpret_cast<float*>(ws + l.off_o);
     p.part_ml = reinterpret_cast<float*>(ws + l.off_ml);
     p.dev_status = dev_status;
+    p.path = (int)desc->flags;
     return launch_verify_attn(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 

@@ -455,6 +455,15 @@ cudaError_t launch_split_d(const AttnParams& p, int mt, const CUtensorMap& mk, c
 
 int attn_rows_pad(int group_rows) { return (group_rows + 15) / 16 * 16; }
 
+// Which split kernel runs.  The warp-MMA kernel re-reads every K/V tile from shared memory once
+// per 16 query rows, which saturates the shared-memory pipe from about 48 rows up; the tcgen05
+// kernel reads each tile once whatever the row count.
+bool attn_use_umma(const AttnParams& p) {
+    if (p.path == 1 || !attn_umma_supported(p)) return false;
+    if (p.path == 2) return true;
+    return attn_rows_pad((p.Hq / p.Hkv) * p.R) >= 48;
+}
+
 cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
     if (p.kv_chunk % kChunkAlign != 0 || p.kv_chunk > kMaxChunkPages * kPageSize) return cudaErrorInvalidValue;
     CUtensorMap mk, mv;
@@ -465,11 +474,15 @@ cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
     const int rows = (p.Hq / p.Hkv) * p.R;
     const int mt = attn_rows_pad(rows) / 16;
     cudaError_t e;
-    switch (p.d) {
-        case 64: e = launch_split_d<64>(p, mt, mk, mv, stream); break;
-        case 128: e = launch_split_d<128>(p, mt, mk, mv, stream); break;
-        case 256: e = launch_split_d<256>(p, mt, mk, mv, stream); break;
-        default: return cudaErrorInvalidValue;
+    if (attn_use_umma(p)) {
+        e = launch_attn_umma(p, mk, mv, stream);
+    } else {
+        switch (p.d) {
+            case 64: e = launch_split_d<64>(p, mt, mk, mv, stream); break;
+            case 128: e = launch_split_d<128>(p, mt, mk, mv, stream); break;
+            case 256: e = launch_split_d<256>(p, mt, mk, mv, stream); break;
+            default: return cudaErrorInvalidValue;
+        }
     }
     if (e != cudaSuccess) return e;
     int launched = 1;

@@ -1,6 +1,8 @@
 // Internal launch interfaces between the C ABI (api.cu) and the kernels.
 #pragma once
 
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace massv {
@@ -21,9 +23,14 @@ struct AttnParams {
     float* part_o;     // [B, Hkv, max_chunks, rows_pad, d] unnormalised partial outputs
     float* part_ml;    // [B, Hkv, max_chunks, rows_pad, 2] running max (log2 domain) and sum
     int32_t* dev_status;
+    int path;          // 0: choose by shape, 1: warp-level MMA kernel, 2: tcgen05 kernel
 };
 int attn_rows_pad(int group_rows);                 // query rows per KV head, padded to the MMA tile
 cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream);
+// tcgen05 variant of the split kernel (attn_umma.cu); the tensor maps are the ones the warp-MMA kernel uses
+bool attn_umma_supported(const AttnParams& p);
+bool attn_use_umma(const AttnParams& p);
+cudaError_t launch_attn_umma(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream);
 
 // ---------------------------------------------------------------- LM head
 struct LmHeadParams {

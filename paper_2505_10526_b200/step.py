@@ -18,12 +18,12 @@ STEP_INPUTS = ("q", "k_new", "v_new", "hidden", "draft_tokens", "draft_probs", "
 class VerifyStep:
     def __init__(self, batch, gamma, n_q_heads, n_kv_heads, head_dim, hidden, vocab, temperature,
                  max_pages_per_seq, num_pages, device="cuda", kv_chunk=0, scale=0.0, window=0,
-                 want_logits=False, want_probs=False, want_attn_f32=False):
+                 attn_kernel=0, want_logits=False, want_probs=False, want_attn_f32=False):
         self.device = torch.device(device)
         self.B, self.gamma, self.R = batch, gamma, gamma + 1
         self.T = float(temperature)
         self.adesc = mv.attn_desc(batch, gamma, n_q_heads, n_kv_heads, head_dim, max_pages_per_seq, num_pages,
-                                  scale=scale, kv_chunk=kv_chunk, window=window)
+                                  scale=scale, kv_chunk=kv_chunk, window=window, kernel=attn_kernel)
         self.cdesc = mv.accept_desc(batch, gamma, hidden, vocab, temperature)
         dev = self.device
         self.attn_ws = mv.alloc_workspace(mv.massv_verify_attn_workspace_size(self.adesc), dev)

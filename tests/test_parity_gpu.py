@@ -219,6 +219,71 @@ def test_odd_shapes_and_forced_splits(spec, kv_chunk):
     run_case(None, cfg=cfg, kv_chunk=kv_chunk)
 
 
+KERNELS = [pytest.param(1, id="warp_mma"), pytest.param(2, id="tcgen05")]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("name,kv_chunk", [("tiny_t1", 0), ("tiny_t1", 64), ("tiny_ragged_t0", 0), ("tiny_ragged_t0", 64),
+                                           ("tiny_ragged_t1", 128), ("tiny_peaked_t1", 64)])
+def test_either_attention_kernel_on_tiny_configs(name, kv_chunk, kernel):
+    """The warp-MMA and the tcgen05 split kernels are interchangeable: each is forced in turn (the
+    library would otherwise pick one by the row count) and held to the same tolerances, with whole
+    contexts in one chunk and with chunks short enough that block rows straddle a chunk boundary."""
+    run_case(name, kv_chunk=kv_chunk, attn_kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("spec", ODD_SHAPES, ids=[s["name"] for s in ODD_SHAPES])
+@pytest.mark.parametrize("kv_chunk", [0, 64])
+def test_either_attention_kernel_on_odd_shapes(spec, kv_chunk, kernel):
+    from workloads import VerifyConfig
+    cfg = VerifyConfig(image_tokens=0.25, draft_noise_std=0.7, seed=40 + len(spec["name"]), **spec)
+    run_case(None, cfg=cfg, kv_chunk=kv_chunk, attn_kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("name,window,kv_chunk,subset", [
+    ("tiny_ragged_t1", 1, 0, None), ("tiny_ragged_t1", 5, 64, None), ("tiny_ragged_t0", 40, 64, None), ("tiny_t1", 100, 64, None),
+    ("qwen7b_b16_t1", 1500, 256, [0, 5, 15]),
+])
+def test_either_attention_kernel_with_a_sliding_window(name, window, kv_chunk, subset, kernel):
+    run_case(name, subset=subset, check_determinism=False, window=window, kv_chunk=kv_chunk, attn_kernel=kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("name,subset", [("qwen7b_b16_t1", [0, 5, 15]), ("gemma12b_b32_t1", [0, 31]), ("qwen7b_long_g7_t0", [0, 63]),
+                                         ("qwen7b_long_g3_t0", [33])])
+def test_either_attention_kernel_at_full_size(name, subset, kernel):
+    run_case(name, subset=subset, check_determinism=False, attn_kernel=kernel)
+
+
+def test_tcgen05_attention_rescales_when_the_maximum_grows():
+    """Scores that keep growing along the context (keys scaled up with position) force the tcgen05
+    kernel to move its reference maximum, i.e. to rescale the accumulator in tensor memory, many
+    times; the result must still be the plain softmax."""
+    from dataclasses import replace
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = replace(get_config("tiny_ragged_t0"), name="growing_scores", batch=3, ctx_lo=700, ctx_hi=900, gamma=7)
+    w = generate(cfg, device="cuda")
+    # q = +1 everywhere, keys grow linearly with the page index they sit in: position i scores about i / 8
+    pt = w["page_table"].long()
+    ramp = torch.zeros(w["k_pages"].shape[0], device="cuda")
+    for b in range(cfg.batch):
+        ramp[pt[b]] = torch.arange(pt.shape[1], device="cuda", dtype=torch.float32)
+    w["q"] = torch.ones_like(w["q"])
+    w["k_pages"] = (torch.ones_like(w["k_pages"].float()) * ramp[:, None, None, None] * (16.0 / 8.0 / 8.0)).to(torch.bfloat16)
+    for kernel in (1, 2):
+        ww = {k: v.clone() for k, v in w.items()}
+        ref = oracle.verify_step({k: v.clone() for k, v in ww.items()}, 0.0)
+        step = VerifyStep.for_workload(cfg, ww, want_attn_f32=True, attn_kernel=kernel, kv_chunk=1024)
+        step.attn(ww)
+        torch.cuda.synchronize()
+        assert int(step.dev_status.item()) == 0
+        err = float(np.abs(step.attn_out_f32.cpu().double().numpy() - ref["attn_out"]).max())
+        lse_err = float(np.abs(step.lse.cpu().double().numpy() - ref["lse"]).max())
+        assert err < TOL_ATTN_F32 and lse_err < TOL_LSE, (kernel, err, lse_err)
+
+
 @pytest.mark.parametrize("name,window,kv_chunk,subset", [
     ("tiny_ragged_t1", 1, 0, None), ("tiny_ragged_t1", 5, 64, None), ("tiny_ragged_t0", 40, 64, None),
     ("tiny_t1", 100, 64, None), ("tiny_t1", 1000, 0, None),
