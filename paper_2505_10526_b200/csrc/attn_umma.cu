@@ -72,15 +72,21 @@ struct UmmaAttnCfg {
     static constexpr int kNCH = D / 64;                       // 64-element column groups of a K/V row
     static constexpr int kRegion = TILE * 128;                // bytes of one (TILE tokens x 64 elements) region
     static constexpr int kEntryBytes = kNCH * kRegion;        // one K tile or one V tile
-    static constexpr int kEntries = 4;                        // ring entries, K and V tiles alternating
+    static constexpr int kEntries = 5;                        // ring entries, filled in the order the MMAs consume them
     static constexpr int kQRegion = kUmmaRows * 128;          // (64 rows x 64 elements)
     static constexpr int kQBytes = kNCH * kQRegion;
     static constexpr int kPBytes = (TILE / 64) * kQRegion;    // P tile: 64 rows x TILE tokens, K-major
-    static constexpr int kSmem = kEntries * kEntryBytes + kQBytes + 2 * kPBytes + 1024;
+    static constexpr int kSmem = kEntries * kEntryBytes + kQBytes + kPBytes + 1024;
     static constexpr int kColsNeeded = 2 * TILE + D;          // two S buffers and O
     static constexpr int kTmemCols = kColsNeeded <= 256 ? 256 : 512;
     static constexpr int kCtasPerSm = (kSmem <= 110 * 1024 && kTmemCols <= 256) ? 2 : 1;
 };
+
+// The MMA thread consumes tiles in the order K_0, K_1, V_0, K_2, V_1, ..., K_{n-1}, V_{n-2}, V_{n-1}
+// (the score product runs two tiles ahead of the softmax).  The ring is filled in the same order,
+// so an entry is never held by a tile that is not needed yet.
+__device__ __forceinline__ int ring_item_of_k(int t) { return t == 0 ? 0 : 2 * t - 1; }
+__device__ __forceinline__ int ring_item_of_v(int t, int n_tiles) { return t == n_tiles - 1 ? 2 * n_tiles - 1 : 2 * t + 2; }
 
 template <int D, int TILE>
 __global__ void __launch_bounds__(kUmmaThreads, UmmaAttnCfg<D, TILE>::kCtasPerSm)
@@ -96,8 +102,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     __shared__ __align__(8) uint64_t landed_bar[E];    // TMA bytes of a tile that still needs patching
     __shared__ __align__(8) uint64_t empty_bar[E];     // the MMAs that read the entry are done
     __shared__ __align__(8) uint64_t s_full_bar[2];    // S buffer written by Q K^T
-    __shared__ __align__(8) uint64_t p_full_bar[2];    // P buffer written (and S buffer read) by the four softmax warps
-    __shared__ __align__(8) uint64_t pv_done_bar[2];   // P V of a tile done: P buffer reusable, O up to date
+    __shared__ __align__(8) uint64_t p_full_bar[2];    // P written (and the S buffer read) by the four softmax warps
+    __shared__ __align__(8) uint64_t pv_done_bar[2];   // P V of a tile done: P may be overwritten, O is up to date
     __shared__ int s_pages[kUmmaMaxChunkPages];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -126,7 +132,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* q_smem = smem + E * Cfg::kEntryBytes;               // [NCH][64 rows][128 B], swizzled
-    uint8_t* p_smem = q_smem + Cfg::kQBytes;                     // 2 x [TILE/64][64 rows][128 B], swizzled
+    uint8_t* p_smem = q_smem + Cfg::kQBytes;                     // [TILE/64][64 rows][128 B], swizzled
 
     if (threadIdx.x == 0) {
         for (int e = 0; e < E; ++e) { mbar_init(&ready_bar[e], 1); mbar_init(&landed_bar[e], 1); mbar_init(&empty_bar[e], 1); }
@@ -169,7 +175,10 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
         uint32_t landed_phase = 0;       // bit e: parity of the next completion of landed_bar[e]
         for (int i = 0; i < 2 * n_tiles; ++i) {
-            const int t = i >> 1, is_v = i & 1, e = i % E;
+            // item i of the consumption order: which tile, and whether its K or its V
+            const int is_v = (i == 2 * n_tiles - 1) || (i > 0 && (i & 1) == 0);
+            const int t = i == 0 ? 0 : (i == 2 * n_tiles - 1 ? n_tiles - 1 : (is_v ? i / 2 - 1 : (i + 1) / 2));
+            const int e = i % E;
             int freed = 0;
             if (lane == 0) freed = mbar_wait(&empty_bar[e], (((uint32_t)(i / E)) & 1u) ^ 1u, abort_ptr) ? 1 : 0;
             freed = __shfl_sync(0xffffffffu, freed, 0);
@@ -233,7 +242,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             bool ok = true;
             // S[t & 1] = Q K_t^T: d/16 steps of 16 elements (32 bytes) along the 128-byte rows
             auto issue_qk = [&](int t) {
-                const int i = 2 * t, e = i % E;
+                const int i = ring_item_of_k(t), e = i % E;
                 if (!mbar_wait(&ready_bar[e], ((uint32_t)(i / E)) & 1u, abort_ptr)) { ok = false; return; }
                 tc_fence_after();
                 const uint32_t k_lo = umma_desc_lo(ring_addr + (uint32_t)e * Cfg::kEntryBytes);
@@ -251,11 +260,11 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             // O (+)= P[t & 1] V_t: TILE/16 steps of 16 tokens; V rows are tokens, so a step is 2048 bytes
             // further and the descriptor's leading offset is the distance between 64-element column groups
             auto issue_pv = [&](int t) {
-                const int i = 2 * t + 1, e = i % E;
+                const int i = ring_item_of_v(t, n_tiles), e = i % E;
                 if (!mbar_wait(&ready_bar[e], ((uint32_t)(i / E)) & 1u, abort_ptr)) { ok = false; return; }
                 if (!mbar_wait(&p_full_bar[t & 1], ((uint32_t)(t >> 1)) & 1u, abort_ptr)) { ok = false; return; }
                 tc_fence_after();
-                const uint32_t p_lo = umma_desc_lo(smem_u32(p_smem) + (uint32_t)((t & 1) * Cfg::kPBytes));
+                const uint32_t p_lo = umma_desc_lo(smem_u32(p_smem));
                 const uint32_t v_lo = (((ring_addr + (uint32_t)e * Cfg::kEntryBytes) & 0x3FFFFu) >> 4) | ((uint32_t)(Cfg::kRegion >> 4) << 16);
 #pragma unroll
                 for (int ks = 0; ks < TILE / 16; ++ks) {
@@ -324,10 +333,24 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             else if (mx0 > m_ref[0] + kRescaleThreshold) { f0 = exp2f(m_ref[0] - mx0); m_ref[0] = mx0; grow = true; }
             if (m_ref[1] == -INFINITY) m_ref[1] = mx1;
             else if (mx1 > m_ref[1] + kRescaleThreshold) { f1 = exp2f(m_ref[1] - mx1); m_ref[1] = mx1; grow = true; }
+            const float ms0 = m_ref[0] == -INFINITY ? 0.f : m_ref[0], ms1 = m_ref[1] == -INFINITY ? 0.f : m_ref[1];
+            float ls0 = 0.f, ls1 = 0.f;
+            uint32_t pk[TILE / 64][16];       // bf16 pairs: [2k] = row r0, [2k+1] = row r1, tokens 8k + 2*(lane%4) + {0,1}
+#pragma unroll
+            for (int h = 0; h < TILE / 64; ++h) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const float p0 = exp2f(__uint_as_float(s[h][4 * k + 0]) - ms0), p1 = exp2f(__uint_as_float(s[h][4 * k + 1]) - ms0);
+                    const float p2 = exp2f(__uint_as_float(s[h][4 * k + 2]) - ms1), p3 = exp2f(__uint_as_float(s[h][4 * k + 3]) - ms1);
+                    ls0 += p0 + p1; ls1 += p2 + p3;
+                    pk[h][2 * k] = pack_bf16x2(p0, p1);
+                    pk[h][2 * k + 1] = pack_bf16x2(p2, p3);
+                }
+            }
+            // P and O belong to the tensor core until P V of tile t-1 is done; P V of tile t cannot
+            // start before this warp has published P below.
+            if (t >= 1 && !mbar_wait_warp(&pv_done_bar[(t - 1) & 1], ((uint32_t)((t - 1) >> 1)) & 1u, abort_ptr)) { ok = false; break; }
             if (__any_sync(0xffffffffu, grow)) {
-                // O holds the products of tiles 0 .. t-1 once P V of tile t-1 is done; P V of tile t
-                // cannot start before this warp has published P below.
-                if (!mbar_wait_warp(&pv_done_bar[(t - 1) & 1], ((uint32_t)((t - 1) >> 1)) & 1u, abort_ptr)) { ok = false; break; }
                 tc_fence_after();
 #pragma unroll 1
                 for (int c0 = 0; c0 < D; c0 += 64) {
@@ -345,21 +368,13 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                 asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
                 l_run[0] *= f0; l_run[1] *= f1;
             }
-            const float ms0 = m_ref[0] == -INFINITY ? 0.f : m_ref[0], ms1 = m_ref[1] == -INFINITY ? 0.f : m_ref[1];
-            // the P buffer is free once P V of tile t-2 has read it
-            if (t >= 2 && !mbar_wait_warp(&pv_done_bar[buf], (((uint32_t)(t >> 1)) & 1u) ^ 1u, abort_ptr)) { ok = false; break; }
-            uint8_t* p_buf = p_smem + buf * Cfg::kPBytes;
-            float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
             for (int h = 0; h < TILE / 64; ++h) {
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const float p0 = exp2f(__uint_as_float(s[h][4 * k + 0]) - ms0), p1 = exp2f(__uint_as_float(s[h][4 * k + 1]) - ms0);
-                    const float p2 = exp2f(__uint_as_float(s[h][4 * k + 2]) - ms1), p3 = exp2f(__uint_as_float(s[h][4 * k + 3]) - ms1);
-                    ls0 += p0 + p1; ls1 += p2 + p3;
                     // tokens 8k .. 8k+7 of the 64-token group are 16-byte unit k of the row
-                    *reinterpret_cast<uint32_t*>(p_buf + h * Cfg::kQRegion + swz128(r0, k) + 4 * (lane & 3)) = pack_bf16x2(p0, p1);
-                    *reinterpret_cast<uint32_t*>(p_buf + h * Cfg::kQRegion + swz128(r1, k) + 4 * (lane & 3)) = pack_bf16x2(p2, p3);
+                    *reinterpret_cast<uint32_t*>(p_smem + h * Cfg::kQRegion + swz128(r0, k) + 4 * (lane & 3)) = pk[h][2 * k];
+                    *reinterpret_cast<uint32_t*>(p_smem + h * Cfg::kQRegion + swz128(r1, k) + 4 * (lane & 3)) = pk[h][2 * k + 1];
                 }
             }
             l_run[0] += ls0; l_run[1] += ls1;
