@@ -52,7 +52,7 @@ int check_attn_desc(const massv_attn_desc* d) {
 
 struct AttnLayout {
     int kv_chunk, max_chunks, rows_pad;
-    size_t off_o, off_ml, total;
+    size_t off_o, off_ml, off_flat_o, off_flat_ml, off_flat_meta, total;
 };
 
 AttnLayout attn_layout(const massv_attn_desc& d) {
@@ -64,7 +64,11 @@ AttnLayout attn_layout(const massv_attn_desc& d) {
     const size_t items = (size_t)d.batch * d.n_kv_heads * l.max_chunks;
     l.off_o = 0;
     l.off_ml = align_up(items * l.rows_pad * d.head_dim * sizeof(float), kAlign);
-    l.total = l.off_ml + align_up(items * l.rows_pad * 2 * sizeof(float), kAlign);
+    l.off_flat_o = l.off_ml + align_up(items * l.rows_pad * 2 * sizeof(float), kAlign);
+    const size_t slots = (size_t)kFlatMaxCtas * 2;
+    l.off_flat_ml = l.off_flat_o + align_up(slots * l.rows_pad * d.head_dim * sizeof(float), kAlign);
+    l.off_flat_meta = l.off_flat_ml + align_up(slots * l.rows_pad * 2 * sizeof(float), kAlign);
+    l.total = l.off_flat_meta + align_up((size_t)(kFlatMaxBatchMeta + 3) * sizeof(int32_t), kAlign);
     return l;
 }
 
@@ -142,6 +146,10 @@ int massv_verify_attn(const massv_attn_desc* desc, const void* q, const void* k_
     p.part_ml = reinterpret_cast<float*>(ws + l.off_ml);
     p.dev_status = dev_status;
     p.path = (int)desc->flags;
+    p.chunk_forced = desc->kv_chunk > 0;
+    p.flat_part_o = reinterpret_cast<float*>(ws + l.off_flat_o);
+    p.flat_part_ml = reinterpret_cast<float*>(ws + l.off_flat_ml);
+    p.flat_meta = reinterpret_cast<int32_t*>(ws + l.off_flat_meta);
     return launch_verify_attn(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 

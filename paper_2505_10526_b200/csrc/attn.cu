@@ -475,7 +475,14 @@ cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
     const int mt = attn_rows_pad(rows) / 16;
     cudaError_t e;
     if (attn_use_umma(p)) {
-        e = launch_attn_umma(p, mk, mv, stream);
+        const bool flat = !p.chunk_forced && attn_umma_flat_supported(p);
+        int launched = 0;
+        e = launch_attn_umma(p, mk, mv, stream, flat, &launched);
+        if (e != cudaSuccess) return e;
+        if (flat) {
+            count_launches(launched);
+            return cudaGetLastError();
+        }
     } else {
         switch (p.d) {
             case 64: e = launch_split_d<64>(p, mt, mk, mv, stream); break;

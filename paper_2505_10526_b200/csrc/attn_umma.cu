@@ -19,7 +19,14 @@
 // as bf16 into shared memory for the second product.  O is rescaled in tensor memory
 // only when a row's running maximum has grown by more than 2^8 since its reference
 // was set (the reference cancels in O / l, so the result is the plain softmax).
-// Sequences that span several chunks are merged by attn_combine_kernel.
+//
+// Two schedules share the kernel.  CHUNKED: grid (chunk, KV head, sequence) as in the warp-MMA
+// kernel, one piece of work per CTA, pieces of a sequence merged by attn_combine_kernel (used
+// when the caller fixes kv_chunk).  FLAT: the tiles of all (sequence, KV head) pairs form one
+// line, ordered by (sequence, head, position); a persistent grid of resident CTAs cuts the line
+// into equal ranges, so every CTA streams the same number of bytes whatever the mix of context
+// lengths, pays its set-up once, and leaves at most two partial results (a pair that began in an
+// earlier CTA, a pair that continues in the next one) to attn_flat_combine_kernel.
 #include "kernels.cuh"
 #include "ptx.cuh"
 #include "umma.cuh"
@@ -31,6 +38,7 @@ namespace {
 constexpr int kUmmaRows = 64;          // MMA M: query rows per KV head, padded
 constexpr int kUmmaThreads = 192;      // producer warp, MMA warp, four softmax warps
 constexpr int kUmmaMaxChunkPages = 256;
+constexpr int kFlatMaxBatch = 1024;    // sequences the flat schedule can index in shared memory
 constexpr float kRescaleThreshold = 8.f;   // log2 units
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -82,13 +90,36 @@ struct UmmaAttnCfg {
     static constexpr int kCtasPerSm = (kSmem <= 110 * 1024 && kTmemCols <= 256) ? 2 : 1;
 };
 
-// The MMA thread consumes tiles in the order K_0, K_1, V_0, K_2, V_1, ..., K_{n-1}, V_{n-2}, V_{n-1}
-// (the score product runs two tiles ahead of the softmax).  The ring is filled in the same order,
-// so an entry is never held by a tile that is not needed yet.
-__device__ __forceinline__ int ring_item_of_k(int t) { return t == 0 ? 0 : 2 * t - 1; }
-__device__ __forceinline__ int ring_item_of_v(int t, int n_tiles) { return t == n_tiles - 1 ? 2 * n_tiles - 1 : 2 * t + 2; }
+// The MMA thread consumes tiles in the order K_0, K_1, K_2, V_0, K_3, V_1, ..., K_{n-1}, V_{n-3}, V_{n-2}, V_{n-1}:
+// the score product of tile t+2 is issued as soon as the softmax warps have read S of tile t (it reuses
+// that buffer), the second product of tile t once they have written P.  The ring is filled in the same
+// order, so an entry is never held by a tile that is not needed yet.
+__device__ __forceinline__ int ring_item_of_k(int t) { return t < 2 ? t : 2 * t - 2; }
+__device__ __forceinline__ int ring_item_of_v(int t, int n_tiles) { return t >= n_tiles - 2 ? 2 * n_tiles - 2 + (t - (n_tiles - 2)) : 3 + 2 * t; }
+// Inverse: item i of a segment of n tiles -> tile index, and whether it is the tile's V.
+__device__ __forceinline__ void ring_item_decode(int i, int n, int& t, int& is_v) {
+    if (n == 1) { t = 0; is_v = i; }
+    else if (i < 2) { t = i; is_v = 0; }
+    else if (i >= 2 * n - 2) { t = n - 2 + (i - (2 * n - 2)); is_v = 1; }
+    else { const int j = i - 2; is_v = j & 1; t = is_v ? (j - 1) / 2 : 2 + j / 2; }
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
-template <int D, int TILE>
+// One piece of work: a run of tiles of one (sequence, KV head) pair.
+struct Segment {
+    int b, g;
+    int L;               // committed length of the sequence
+    int c_begin, c_end;  // token range [c_begin, c_end), c_begin a multiple of TILE
+    int n_tiles;
+    float* part_o;       // where the unnormalised partial result goes; nullptr: the piece is the whole pair
+    float* part_ml;
+};
+
+template <int D, int TILE, bool FLAT>
 __global__ void __launch_bounds__(kUmmaThreads, UmmaAttnCfg<D, TILE>::kCtasPerSm)
 attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
     using Cfg = UmmaAttnCfg<D, TILE>;
@@ -96,39 +127,137 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     constexpr int NCH = Cfg::kNCH;
     constexpr int UPR = D / 8;             // 16-byte units per K/V/Q row
     constexpr int PPT = TILE / kPageSize;  // pages per tile
+    constexpr int GROUP = 32 / PPT;        // tiles whose page ids fit one register per lane
+    static_assert(PPT * NCH <= 32 && GROUP >= 3, "one TMA box per lane; V tiles trail K tiles by at most three");
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t ready_bar[E];     // tile complete (landed, and patched where needed)
     __shared__ __align__(8) uint64_t landed_bar[E];    // TMA bytes of a tile that still needs patching
     __shared__ __align__(8) uint64_t empty_bar[E];     // the MMAs that read the entry are done
     __shared__ __align__(8) uint64_t s_full_bar[2];    // S buffer written by Q K^T
-    __shared__ __align__(8) uint64_t p_full_bar[2];    // P written (and the S buffer read) by the four softmax warps
+    __shared__ __align__(8) uint64_t s_read_bar[2];    // S buffer copied to registers by the four softmax warps
+    __shared__ __align__(8) uint64_t p_full_bar[2];    // P written by the four softmax warps
     __shared__ __align__(8) uint64_t pv_done_bar[2];   // P V of a tile done: P may be overwritten, O is up to date
-    __shared__ int s_pages[kUmmaMaxChunkPages];
+    __shared__ __align__(8) uint64_t q_ready_bar;      // the query rows of the next segment are in shared memory
+    __shared__ int s_cum[FLAT ? kFlatMaxBatch + 1 : 1];   // FLAT: tiles of sequences 0 .. b-1 (per KV head)
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
-    const int chunk = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    pdl_wait();
-    const int L = p.seq_lens[b];
-    if (L < 0 || L + p.R > p.max_pages * kPageSize) {            // no room for the block: skip the sequence
-        if (chunk == 0 && g == 0 && threadIdx.x == 0) set_status(p.dev_status, MASSV_ERR_CAPACITY);
-        return;
-    }
-    const int n_ctx = L + p.R;
-    if (chunk * p.kv_chunk >= n_ctx) return;
-    // Sliding window: nothing before block row 0's lower bound is needed (see the warp-MMA kernel).
-    const int lo_min = p.window > 0 ? max(0, L - p.window + 1) : 0;
-    const int first_chunk = lo_min / p.kv_chunk;
-    if (chunk < first_chunk) return;
-    int c_begin = chunk * p.kv_chunk;
-    if (chunk == first_chunk) c_begin += ((lo_min - c_begin) / TILE) * TILE;
-    const int c_end = min(n_ctx, chunk * p.kv_chunk + p.kv_chunk);
-    const int n_tiles = (c_end - c_begin + TILE - 1) / TILE;
-    const int n_chunks_b = (n_ctx + p.kv_chunk - 1) / p.kv_chunk - first_chunk;
     const int G = p.Hq / p.Hkv;
     const int rows = G * p.R;
+    const int rows_pad = (rows + 15) / 16 * 16;
+    pdl_wait();
+
+    // ---------------------------------------------------- this CTA's share of the work
+    int f = 0, f_end = 0;                 // FLAT: range of the tile line; CHUNKED: one pseudo-tile
+    if constexpr (FLAT) {
+        // tiles per pair of every sequence, then an exclusive prefix sum over the batch
+        for (int i = threadIdx.x; i < p.B; i += blockDim.x) {
+            const int L = p.seq_lens[i];
+            int n = 0;
+            if (L < 0 || L + p.R > p.max_pages * kPageSize) {       // no room for the block: skip the sequence
+                if (blockIdx.x == 0) set_status(p.dev_status, MASSV_ERR_CAPACITY);
+            } else {
+                const int lo_min = p.window > 0 ? max(0, L - p.window + 1) : 0;
+                n = (L + p.R + TILE - 1) / TILE - lo_min / TILE;
+            }
+            s_cum[i + 1] = n;
+        }
+        if (threadIdx.x == 0) s_cum[0] = 0;
+        __syncthreads();
+        if (warp == 0) {
+            const int per = (p.B + 31) / 32;
+            const int i0 = min(p.B, lane * per), i1 = min(p.B, i0 + per);
+            int local = 0;
+            for (int i = i0; i < i1; ++i) local += s_cum[i + 1];
+            int incl = local;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            int run = incl - local;
+            for (int i = i0; i < i1; ++i) { run += s_cum[i + 1]; s_cum[i + 1] = run; }
+        }
+        __syncthreads();
+        const int total = s_cum[p.B] * p.Hkv;
+        const int per_cta = max(1, (total + (int)gridDim.x - 1) / (int)gridDim.x);
+        if (blockIdx.x == 0) {      // what the merge kernel needs to find the pieces of a pair
+            for (int i = threadIdx.x; i <= p.B; i += blockDim.x) p.flat_meta[2 + i] = s_cum[i];
+            if (threadIdx.x == 0) { p.flat_meta[0] = per_cta; p.flat_meta[1] = total; }
+        }
+        f = min(total, (int)blockIdx.x * per_cta);
+        f_end = min(total, f + per_cta);
+        if (f >= f_end) return;
+    } else {
+        const int b = blockIdx.z, chunk = blockIdx.x;
+        const int L = p.seq_lens[b];
+        if (L < 0 || L + p.R > p.max_pages * kPageSize) {
+            if (chunk == 0 && blockIdx.y == 0 && threadIdx.x == 0) set_status(p.dev_status, MASSV_ERR_CAPACITY);
+            return;
+        }
+        if (chunk * p.kv_chunk >= L + p.R) return;
+        const int lo_min = p.window > 0 ? max(0, L - p.window + 1) : 0;
+        if (chunk < lo_min / p.kv_chunk) return;
+        f = 0; f_end = 1;
+    }
+    const int f_first = f;
+    int b_hint = 0;
+    // Next piece of this CTA's share; false when the share is used up.
+    auto next_segment = [&](Segment& sg) -> bool {
+        if (f >= f_end) return false;
+        if constexpr (FLAT) {
+            // the sequence whose pairs hold tile f of the line: largest b with Hkv * cum[b] <= f
+            int lo = b_hint, hi = p.B - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (s_cum[mid] * p.Hkv <= f) lo = mid; else hi = mid - 1;
+            }
+            b_hint = lo;
+            const int n_b = s_cum[lo + 1] - s_cum[lo];
+            const int off = f - s_cum[lo] * p.Hkv;
+            const int g = off / n_b, t0 = off % n_b, t1 = min(n_b, t0 + (f_end - f));
+            const int L = p.seq_lens[lo];
+            const int tile_lo = (p.window > 0 ? max(0, L - p.window + 1) : 0) / TILE;
+            sg.b = lo; sg.g = g; sg.L = L;
+            sg.c_begin = (tile_lo + t0) * TILE;
+            sg.c_end = min(L + p.R, (tile_lo + t1) * TILE);
+            sg.n_tiles = t1 - t0;
+            if (t0 == 0 && t1 == n_b) {
+                sg.part_o = nullptr; sg.part_ml = nullptr;
+            } else {
+                // slot 0: the piece that opens this CTA's range; slot 1: a later piece (it can only be
+                // one that runs on into the next CTA)
+                const size_t slot = (size_t)blockIdx.x * 2 + (f == f_first ? 0 : 1);
+                sg.part_o = p.flat_part_o + slot * rows_pad * D;
+                sg.part_ml = p.flat_part_ml + slot * rows_pad * 2;
+            }
+            f += t1 - t0;
+        } else {
+            const int b = blockIdx.z, g = blockIdx.y, chunk = blockIdx.x;
+            const int L = p.seq_lens[b];
+            const int n_ctx = L + p.R;
+            const int lo_min = p.window > 0 ? max(0, L - p.window + 1) : 0;
+            const int first_chunk = lo_min / p.kv_chunk;
+            int c_begin = chunk * p.kv_chunk;
+            if (chunk == first_chunk) c_begin += ((lo_min - c_begin) / TILE) * TILE;
+            sg.b = b; sg.g = g; sg.L = L;
+            sg.c_begin = c_begin;
+            sg.c_end = min(n_ctx, chunk * p.kv_chunk + p.kv_chunk);
+            sg.n_tiles = (sg.c_end - c_begin + TILE - 1) / TILE;
+            const int n_chunks_b = (n_ctx + p.kv_chunk - 1) / p.kv_chunk - first_chunk;
+            if (n_chunks_b == 1) {
+                sg.part_o = nullptr; sg.part_ml = nullptr;
+            } else {
+                const size_t item = ((size_t)b * p.Hkv + g) * p.max_chunks + chunk;
+                sg.part_o = p.part_o + item * rows_pad * D;
+                sg.part_ml = p.part_ml + item * rows_pad * 2;
+            }
+            f = f_end;
+        }
+        return true;
+    };
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* q_smem = smem + E * Cfg::kEntryBytes;               // [NCH][64 rows][128 B], swizzled
@@ -136,7 +265,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
 
     if (threadIdx.x == 0) {
         for (int e = 0; e < E; ++e) { mbar_init(&ready_bar[e], 1); mbar_init(&landed_bar[e], 1); mbar_init(&empty_bar[e], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&s_full_bar[i], 1); mbar_init(&p_full_bar[i], 4); mbar_init(&pv_done_bar[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&s_full_bar[i], 1); mbar_init(&s_read_bar[i], 4); mbar_init(&p_full_bar[i], 4); mbar_init(&pv_done_bar[i], 1); }
+        mbar_init(&q_ready_bar, 4);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -147,86 +277,99 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    {   // page ids of this chunk and the query rows (row r = block_row * G + head_in_group; rows past the last are zero)
-        const int n_pages = (c_end - c_begin + kPageSize - 1) / kPageSize;
-        for (int i = threadIdx.x; i < n_pages; i += blockDim.x)
-            s_pages[i] = p.page_table[(size_t)b * p.max_pages + c_begin / kPageSize + i];
-        for (int i = threadIdx.x; i < kUmmaRows * UPR; i += blockDim.x) {
-            const int r = i / UPR, u = i % UPR;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (r < rows) {
-                const int j = r / G, hh = r % G;
-                v = *reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.R + j) * p.Hq + g * G + hh) * D + u * 8);
-            }
-            *reinterpret_cast<uint4*>(q_smem + (u / 8) * Cfg::kQRegion + swz128(r, u % 8)) = v;
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // Q is read by the tensor core
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t tmem_o = tmem_base + 2 * TILE;
     volatile int* abort_ptr = &abort_flag;
+    Segment sg;
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (+ append / ragged-end patch)
         uint64_t policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
         uint32_t landed_phase = 0;       // bit e: parity of the next completion of landed_bar[e]
-        for (int i = 0; i < 2 * n_tiles; ++i) {
-            // item i of the consumption order: which tile, and whether its K or its V
-            const int is_v = (i == 2 * n_tiles - 1) || (i > 0 && (i & 1) == 0);
-            const int t = i == 0 ? 0 : (i == 2 * n_tiles - 1 ? n_tiles - 1 : (is_v ? i / 2 - 1 : (i + 1) / 2));
-            const int e = i % E;
-            int freed = 0;
-            if (lane == 0) freed = mbar_wait(&empty_bar[e], (((uint32_t)(i / E)) & 1u) ^ 1u, abort_ptr) ? 1 : 0;
-            freed = __shfl_sync(0xffffffffu, freed, 0);
-            if (!freed) break;
-            const int tile_start = c_begin + t * TILE;
-            const int valid = min(TILE, c_end - tile_start);
-            const int n_pg = (valid + kPageSize - 1) / kPageSize;
-            const bool patch = tile_start + TILE > L;           // the tile holds block rows or the ragged end
-            uint64_t* bar = patch ? &landed_bar[e] : &ready_bar[e];
-            uint8_t* dst = smem + (size_t)e * Cfg::kEntryBytes;
-            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_pg * NCH * 2048));
-            __syncwarp();
-            for (int j = lane; j < n_pg * NCH; j += 32) {
-                const int dc = j % NCH, pg = j / NCH;
-                int pid = s_pages[t * PPT + pg];
-                if (pid < 0 || pid >= p.num_pages) { set_status(p.dev_status, MASSV_ERR_CAPACITY); pid = 0; }
-                tma_load_2d(dst + dc * Cfg::kRegion + pg * 2048, is_v ? &map_v : &map_k, dc * 64, (pid * p.Hkv + g) * kPageSize, bar, policy);
-            }
-            if (patch) {
-                int ok = 0;
-                if (lane == 0) ok = mbar_wait(&landed_bar[e], (landed_phase >> e) & 1u, abort_ptr) ? 1 : 0;
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) break;
-                landed_phase ^= 1u << e;
-                // The block's rows (positions L .. L+gamma) are not in the cache yet: put them into the
-                // tile and store them to their page slots.
-                const int p_first = max(L, tile_start), p_last = min(c_end, tile_start + TILE);
-                const __nv_bfloat16* src_base = is_v ? p.v_new : p.k_new;
-                __nv_bfloat16* pages = is_v ? p.v_pages : p.k_pages;
-                for (int idx = lane; idx < (p_last - p_first) * UPR; idx += 32) {
-                    const int pos = p_first + idx / UPR, u = idx % UPR, row = pos - tile_start;
-                    const uint4 val = *reinterpret_cast<const uint4*>(src_base + (((size_t)b * p.R + (pos - L)) * p.Hkv + g) * D + u * 8);
-                    *reinterpret_cast<uint4*>(dst + (u / 8) * Cfg::kRegion + swz128(row, u % 8)) = val;
-                    const int pid = s_pages[(pos - c_begin) / kPageSize];
-                    if (pid >= 0 && pid < p.num_pages)
-                        *reinterpret_cast<uint4*>(pages + (((size_t)pid * p.Hkv + g) * kPageSize + (pos % kPageSize)) * D + u * 8) = val;
+        int it = 0;                      // items issued so far: ring entry it % E, use it / E
+        bool ok = true;
+        while (ok && next_segment(sg)) {
+            const int n_tiles = sg.n_tiles, L = sg.L, b = sg.b, g = sg.g;
+            // Page ids travel in registers: lane l holds the id of page 32 * group + l of the segment, for
+            // the group of the most advanced K tile (cur), the one before (prev: V tiles trail K tiles by up
+            // to three tiles) and the one after (next: fetched a whole group ahead, so the table lookup is
+            // never on the critical path).
+            const int32_t* pt = p.page_table + (size_t)b * p.max_pages + sg.c_begin / kPageSize;
+            const int n_pages = (sg.c_end - sg.c_begin + kPageSize - 1) / kPageSize;
+            int pid_prev = 0, pid_cur = lane < n_pages ? pt[lane] : 0, pid_next = 32 + lane < n_pages ? pt[32 + lane] : 0;
+            int grp_cur = 0;
+            for (int i = 0; i < 2 * n_tiles; ++i, ++it) {
+                // item i of the consumption order: which tile, and whether its K or its V
+                int t, is_v;
+                ring_item_decode(i, n_tiles, t, is_v);
+                const int e = it % E;
+                if (t / GROUP > grp_cur) {           // only a K tile can be the first of a new group
+                    grp_cur = t / GROUP;
+                    pid_prev = pid_cur; pid_cur = pid_next;
+                    const int nxt = (grp_cur + 1) * 32 + lane;
+                    pid_next = nxt < n_pages ? pt[nxt] : 0;
                 }
-                if (is_v) {
-                    // rows past the end of the context hold stale bytes; their weights are zero, but
-                    // 0 * NaN would still poison P V
-                    for (int idx = lane; idx < (TILE - valid) * UPR; idx += 32) {
-                        const int row = valid + idx / UPR, u = idx % UPR;
-                        *reinterpret_cast<uint4*>(dst + (u / 8) * Cfg::kRegion + swz128(row, u % 8)) = make_uint4(0u, 0u, 0u, 0u);
-                    }
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                int tile_pid[PPT];                   // ids of this tile's pages
+#pragma unroll
+                for (int pg = 0; pg < PPT; ++pg)
+                    tile_pid[pg] = __shfl_sync(0xffffffffu, t / GROUP == grp_cur ? pid_cur : pid_prev, (t % GROUP) * PPT + pg);
+                int freed = 0;
+                if (lane == 0) freed = mbar_wait(&empty_bar[e], (((uint32_t)(it / E)) & 1u) ^ 1u, abort_ptr) ? 1 : 0;
+                freed = __shfl_sync(0xffffffffu, freed, 0);
+                if (!freed) { ok = false; break; }
+                const int tile_start = sg.c_begin + t * TILE;
+                const int valid = min(TILE, sg.c_end - tile_start);
+                const int n_pg = (valid + kPageSize - 1) / kPageSize;
+                const bool patch = tile_start + TILE > L;           // the tile holds block rows or the ragged end
+                uint64_t* bar = patch ? &landed_bar[e] : &ready_bar[e];
+                uint8_t* dst = smem + (size_t)e * Cfg::kEntryBytes;
+                if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_pg * NCH * 2048));
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&ready_bar[e]);
+                if (lane < n_pg * NCH) {             // one 16-token x 64-element box per lane
+                    const int dc = lane % NCH, pg = lane / NCH;
+                    int pid = tile_pid[0];
+#pragma unroll
+                    for (int q = 1; q < PPT; ++q) pid = pg == q ? tile_pid[q] : pid;
+                    if (pid < 0 || pid >= p.num_pages) { set_status(p.dev_status, MASSV_ERR_CAPACITY); pid = 0; }
+                    tma_load_2d(dst + dc * Cfg::kRegion + pg * 2048, is_v ? &map_v : &map_k, dc * 64, (pid * p.Hkv + g) * kPageSize, bar, policy);
+                }
+                if (patch) {
+                    int landed = 0;
+                    if (lane == 0) landed = mbar_wait(&landed_bar[e], (landed_phase >> e) & 1u, abort_ptr) ? 1 : 0;
+                    landed = __shfl_sync(0xffffffffu, landed, 0);
+                    if (!landed) { ok = false; break; }
+                    landed_phase ^= 1u << e;
+                    // The block's rows (positions L .. L+gamma) are not in the cache yet: put them into the
+                    // tile and store them to their page slots.
+                    const int p_first = max(L, tile_start), p_last = min(sg.c_end, tile_start + TILE);
+                    const __nv_bfloat16* src_base = is_v ? p.v_new : p.k_new;
+                    __nv_bfloat16* pages = is_v ? p.v_pages : p.k_pages;
+                    for (int idx = lane; idx < (p_last - p_first) * UPR; idx += 32) {
+                        const int pos = p_first + idx / UPR, u = idx % UPR, row = pos - tile_start;
+                        const uint4 val = *reinterpret_cast<const uint4*>(src_base + (((size_t)b * p.R + (pos - L)) * p.Hkv + g) * D + u * 8);
+                        *reinterpret_cast<uint4*>(dst + (u / 8) * Cfg::kRegion + swz128(row, u % 8)) = val;
+                        int pid = tile_pid[0];
+#pragma unroll
+                        for (int q = 1; q < PPT; ++q) pid = row / kPageSize == q ? tile_pid[q] : pid;
+                        if (pid >= 0 && pid < p.num_pages)
+                            *reinterpret_cast<uint4*>(pages + (((size_t)pid * p.Hkv + g) * kPageSize + (pos % kPageSize)) * D + u * 8) = val;
+                    }
+                    if (is_v) {
+                        // rows past the end of the context hold stale bytes; their weights are zero, but
+                        // 0 * NaN would still poison P V
+                        for (int idx = lane; idx < (TILE - valid) * UPR; idx += 32) {
+                            const int row = valid + idx / UPR, u = idx % UPR;
+                            *reinterpret_cast<uint4*>(dst + (u / 8) * Cfg::kRegion + swz128(row, u % 8)) = make_uint4(0u, 0u, 0u, 0u);
+                        }
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ready_bar[e]);
+                }
             }
         }
         if (lane == 0 && *abort_ptr) {
@@ -238,15 +381,17 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kUmmaRows, TILE, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(kUmmaRows, D, true);
             const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem));
+            const uint32_t p_lo = umma_desc_lo(smem_u32(p_smem));
             const uint32_t ring_addr = smem_u32(smem);
             bool ok = true;
-            // S[t & 1] = Q K_t^T: d/16 steps of 16 elements (32 bytes) along the 128-byte rows
+            int it_base = 0, tau_base = 0, n_tiles = 0;      // ring items / tiles of earlier segments
+            // S[tau & 1] = Q K_t^T: d/16 steps of 16 elements (32 bytes) along the 128-byte rows
             auto issue_qk = [&](int t) {
-                const int i = ring_item_of_k(t), e = i % E;
+                const int i = it_base + ring_item_of_k(t), e = i % E, tau = tau_base + t;
                 if (!mbar_wait(&ready_bar[e], ((uint32_t)(i / E)) & 1u, abort_ptr)) { ok = false; return; }
                 tc_fence_after();
                 const uint32_t k_lo = umma_desc_lo(ring_addr + (uint32_t)e * Cfg::kEntryBytes);
-                const uint32_t d_tmem = tmem_base + (uint32_t)((t & 1) * TILE);
+                const uint32_t d_tmem = tmem_base + (uint32_t)((tau & 1) * TILE);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t a = q_lo + (uint32_t)(((kk >> 2) * Cfg::kQRegion + (kk & 3) * 32) >> 4);
@@ -255,16 +400,15 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                     else umma_bf16<true>(d_tmem, a, bb, idesc_qk);
                 }
                 umma_commit(&empty_bar[e]);
-                umma_commit(&s_full_bar[t & 1]);
+                umma_commit(&s_full_bar[tau & 1]);
             };
-            // O (+)= P[t & 1] V_t: TILE/16 steps of 16 tokens; V rows are tokens, so a step is 2048 bytes
+            // O (+)= P V_t: TILE/16 steps of 16 tokens; V rows are tokens, so a step is 2048 bytes
             // further and the descriptor's leading offset is the distance between 64-element column groups
             auto issue_pv = [&](int t) {
-                const int i = ring_item_of_v(t, n_tiles), e = i % E;
+                const int i = it_base + ring_item_of_v(t, n_tiles), e = i % E, tau = tau_base + t;
                 if (!mbar_wait(&ready_bar[e], ((uint32_t)(i / E)) & 1u, abort_ptr)) { ok = false; return; }
-                if (!mbar_wait(&p_full_bar[t & 1], ((uint32_t)(t >> 1)) & 1u, abort_ptr)) { ok = false; return; }
+                if (!mbar_wait(&p_full_bar[tau & 1], ((uint32_t)(tau >> 1)) & 1u, abort_ptr)) { ok = false; return; }
                 tc_fence_after();
-                const uint32_t p_lo = umma_desc_lo(smem_u32(p_smem));
                 const uint32_t v_lo = (((ring_addr + (uint32_t)e * Cfg::kEntryBytes) & 0x3FFFFu) >> 4) | ((uint32_t)(Cfg::kRegion >> 4) << 16);
 #pragma unroll
                 for (int ks = 0; ks < TILE / 16; ++ks) {
@@ -274,13 +418,28 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                     else umma_bf16<true>(tmem_o, a, bb, idesc_pv);
                 }
                 umma_commit(&empty_bar[e]);
-                umma_commit(&pv_done_bar[t & 1]);
+                umma_commit(&pv_done_bar[tau & 1]);
             };
-            issue_qk(0);
-            if (ok && n_tiles > 1) issue_qk(1);
-            for (int t = 0; t < n_tiles && ok; ++t) {
-                issue_pv(t);
-                if (ok && t + 2 < n_tiles) issue_qk(t + 2);
+            for (int seg = 0; ok && next_segment(sg); ++seg) {
+                n_tiles = sg.n_tiles;
+                // the softmax warps have read the previous segment's O and written this segment's Q
+                if (!mbar_wait(&q_ready_bar, (uint32_t)seg & 1u, abort_ptr)) { ok = false; break; }
+                tc_fence_after();
+                issue_qk(0);
+                if (ok && n_tiles > 1) issue_qk(1);
+                for (int t = 0; t < n_tiles && ok; ++t) {
+                    if (t + 2 < n_tiles) {
+                        // S of tile t is in the softmax warps' registers: its buffer takes tile t+2.  Issued here,
+                        // the score MMAs run while the softmax computes, and a tcgen05.ld (which queues behind
+                        // the MMAs issued before it) finds only the short second product in front of it.
+                        const int tau = tau_base + t;
+                        if (!mbar_wait(&s_read_bar[tau & 1], ((uint32_t)(tau >> 1)) & 1u, abort_ptr)) { ok = false; break; }
+                        issue_qk(t + 2);
+                    }
+                    if (ok) issue_pv(t);
+                }
+                it_base += 2 * n_tiles;
+                tau_base += n_tiles;
             }
         }
     } else {
@@ -291,109 +450,150 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         // block row of each of this thread's two query rows (padding rows behave like the last block row)
         const int j0 = r0 < rows ? r0 / G : p.R - 1, j1 = r1 < rows ? r1 / G : p.R - 1;
         const float scale_log2 = p.scale * 1.4426950408889634f;
-        float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+        const int sm_tid = threadIdx.x - 64;                // 0 .. 127 among the softmax warps
+        uint8_t* p_row0 = p_smem + r0 * 128 + 4 * (lane & 3);   // this thread's 4 bytes of unit 0 of row r0 (before the swizzle)
         bool ok = true;
-        for (int t = 0; t < n_tiles && ok; ++t) {
-            const int buf = t & 1;
-            if (!mbar_wait_warp(&s_full_bar[buf], ((uint32_t)(t >> 1)) & 1u, abort_ptr)) { ok = false; break; }
-            tc_fence_after();
-            const int tile_start = c_begin + t * TILE;
-            // some position in the tile is hidden from some block row: ahead of row 0, or (with a
-            // window) older than the last row's lower bound
-            const bool need_mask = tile_start + TILE > L + 1 || (p.window > 0 && tile_start < n_ctx - p.window);
-            float mx0 = -INFINITY, mx1 = -INFINITY;
-            uint32_t s[TILE / 64][32];
-#pragma unroll
-            for (int h = 0; h < TILE / 64; ++h) {
-                tmem_ld_16x64(tmem_base + lane_base + (uint32_t)(buf * TILE + h * 64), s[h]);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        float sv = __uint_as_float(s[h][4 * k + e]) * scale_log2;
-                        if (need_mask) {
-                            const int pos = tile_start + h * 64 + k * 8 + 2 * (lane & 3) + (e & 1);
-                            const int row_pos = L + (e < 2 ? j0 : j1);
-                            if (pos > row_pos || (p.window > 0 && pos < row_pos - p.window + 1)) sv = -INFINITY;
-                        }
-                        s[h][4 * k + e] = __float_as_uint(sv);
-                        if (e < 2) mx0 = fmaxf(mx0, sv); else mx1 = fmaxf(mx1, sv);
-                    }
-                }
+        int tau_base = 0;
+        while (ok && next_segment(sg)) {
+            const int L = sg.L, b = sg.b, g = sg.g, n_tiles = sg.n_tiles, n_ctx = L + p.R;
+            // query rows of the pair (row r = block_row * G + head_in_group; rows past the last are zero).
+            // Every MMA that read the previous Q and every read of the previous O is finished by now.
+            for (int i = sm_tid; i < kUmmaRows * UPR; i += 128) {
+                const int r = i / UPR, u = i % UPR;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (r < rows)
+                    v = *reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.R + r / G) * p.Hq + g * G + r % G) * D + u * 8);
+                *reinterpret_cast<uint4*>(q_smem + (u / 8) * Cfg::kQRegion + swz128(r, u % 8)) = v;
             }
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-            // The reference maximum of a row moves only when the row's maximum has outgrown it by the
-            // threshold (or when it is first set); O and l are then rescaled to the new reference.
-            float f0 = 1.f, f1 = 1.f;
-            bool grow = false;
-            if (m_ref[0] == -INFINITY) m_ref[0] = mx0;
-            else if (mx0 > m_ref[0] + kRescaleThreshold) { f0 = exp2f(m_ref[0] - mx0); m_ref[0] = mx0; grow = true; }
-            if (m_ref[1] == -INFINITY) m_ref[1] = mx1;
-            else if (mx1 > m_ref[1] + kRescaleThreshold) { f1 = exp2f(m_ref[1] - mx1); m_ref[1] = mx1; grow = true; }
-            const float ms0 = m_ref[0] == -INFINITY ? 0.f : m_ref[0], ms1 = m_ref[1] == -INFINITY ? 0.f : m_ref[1];
-            float ls0 = 0.f, ls1 = 0.f;
-            uint32_t pk[TILE / 64][16];       // bf16 pairs: [2k] = row r0, [2k+1] = row r1, tokens 8k + 2*(lane%4) + {0,1}
-#pragma unroll
-            for (int h = 0; h < TILE / 64; ++h) {
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float p0 = exp2f(__uint_as_float(s[h][4 * k + 0]) - ms0), p1 = exp2f(__uint_as_float(s[h][4 * k + 1]) - ms0);
-                    const float p2 = exp2f(__uint_as_float(s[h][4 * k + 2]) - ms1), p3 = exp2f(__uint_as_float(s[h][4 * k + 3]) - ms1);
-                    ls0 += p0 + p1; ls1 += p2 + p3;
-                    pk[h][2 * k] = pack_bf16x2(p0, p1);
-                    pk[h][2 * k + 1] = pack_bf16x2(p2, p3);
-                }
-            }
-            // P and O belong to the tensor core until P V of tile t-1 is done; P V of tile t cannot
-            // start before this warp has published P below.
-            if (t >= 1 && !mbar_wait_warp(&pv_done_bar[(t - 1) & 1], ((uint32_t)((t - 1) >> 1)) & 1u, abort_ptr)) { ok = false; break; }
-            if (__any_sync(0xffffffffu, grow)) {
-                tc_fence_after();
-#pragma unroll 1
-                for (int c0 = 0; c0 < D; c0 += 64) {
-                    uint32_t o[32];
-                    tmem_ld_16x64(tmem_o + lane_base + (uint32_t)c0, o);
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        o[4 * k + 0] = __float_as_uint(__uint_as_float(o[4 * k + 0]) * f0);
-                        o[4 * k + 1] = __float_as_uint(__uint_as_float(o[4 * k + 1]) * f0);
-                        o[4 * k + 2] = __float_as_uint(__uint_as_float(o[4 * k + 2]) * f1);
-                        o[4 * k + 3] = __float_as_uint(__uint_as_float(o[4 * k + 3]) * f1);
-                    }
-                    tmem_st_16x64(tmem_o + lane_base + (uint32_t)c0, o);
-                }
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                l_run[0] *= f0; l_run[1] *= f1;
-            }
-#pragma unroll
-            for (int h = 0; h < TILE / 64; ++h) {
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    // tokens 8k .. 8k+7 of the 64-token group are 16-byte unit k of the row
-                    *reinterpret_cast<uint32_t*>(p_smem + h * Cfg::kQRegion + swz128(r0, k) + 4 * (lane & 3)) = pk[h][2 * k];
-                    *reinterpret_cast<uint32_t*>(p_smem + h * Cfg::kQRegion + swz128(r1, k) + 4 * (lane & 3)) = pk[h][2 * k + 1];
-                }
-            }
-            l_run[0] += ls0; l_run[1] += ls1;
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // P is read by the tensor core
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // Q is read by the tensor core
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&p_full_bar[buf]);
-        }
-        if (ok && !mbar_wait_warp(&pv_done_bar[(n_tiles - 1) & 1], ((uint32_t)((n_tiles - 1) >> 1)) & 1u, abort_ptr)) ok = false;
-        tc_fence_after();
-        pdl_trigger();
-        if (ok) {
+            if (lane == 0) mbar_arrive(&q_ready_bar);
+
+            float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int tau = tau_base + t, buf = tau & 1;
+                if (!mbar_wait_warp(&s_full_bar[buf], ((uint32_t)(tau >> 1)) & 1u, abort_ptr)) { ok = false; break; }
+                tc_fence_after();
+                const int tile_start = sg.c_begin + t * TILE;
+                // some position in the tile is hidden from some block row: ahead of row 0, or (with a
+                // window) older than the last row's lower bound
+                const bool need_mask = tile_start + TILE > L + 1 || (p.window > 0 && tile_start < n_ctx - p.window);
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+                uint32_t s[TILE / 64][32];         // raw scores; the scale is applied inside the exponential
+#pragma unroll
+                for (int h = 0; h < TILE / 64; ++h) tmem_ld_16x64(tmem_base + lane_base + (uint32_t)(buf * TILE + h * 64), s[h]);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_read_bar[buf]);        // the buffer may take the scores of tile t+2
+                if (need_mask) {
+                    // only the tiles at the ragged end (and, with a window, at its lower edge) come here
+#pragma unroll
+                    for (int h = 0; h < TILE / 64; ++h) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int pos = tile_start + h * 64 + k * 8 + 2 * (lane & 3) + (e & 1);
+                                const int row_pos = L + (e < 2 ? j0 : j1);
+                                if (pos > row_pos || (p.window > 0 && pos < row_pos - p.window + 1)) s[h][4 * k + e] = 0xff800000u;   // -inf
+                            }
+                        }
+                    }
+                }
+                {
+                    // row maxima with four independent chains per row
+                    float ma[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY}, mb[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int h = 0; h < TILE / 64; ++h) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            ma[k & 3] = fmaxf(ma[k & 3], fmaxf(__uint_as_float(s[h][4 * k + 0]), __uint_as_float(s[h][4 * k + 1])));
+                            mb[k & 3] = fmaxf(mb[k & 3], fmaxf(__uint_as_float(s[h][4 * k + 2]), __uint_as_float(s[h][4 * k + 3])));
+                        }
+                    }
+                    mx0 = fmaxf(fmaxf(ma[0], ma[1]), fmaxf(ma[2], ma[3]));
+                    mx1 = fmaxf(fmaxf(mb[0], mb[1]), fmaxf(mb[2], mb[3]));
+                }
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                mx0 *= scale_log2; mx1 *= scale_log2;             // log2 domain (the scale is positive)
+                // The reference maximum of a row moves only when the row's maximum has outgrown it by the
+                // threshold (or when it is first set); O and l are then rescaled to the new reference.
+                float f0 = 1.f, f1 = 1.f;
+                bool grow = false;
+                if (m_ref[0] == -INFINITY) m_ref[0] = mx0;
+                else if (mx0 > m_ref[0] + kRescaleThreshold) { f0 = exp2f(m_ref[0] - mx0); m_ref[0] = mx0; grow = true; }
+                if (m_ref[1] == -INFINITY) m_ref[1] = mx1;
+                else if (mx1 > m_ref[1] + kRescaleThreshold) { f1 = exp2f(m_ref[1] - mx1); m_ref[1] = mx1; grow = true; }
+                const float ms0 = m_ref[0] == -INFINITY ? 0.f : -m_ref[0], ms1 = m_ref[1] == -INFINITY ? 0.f : -m_ref[1];
+                float la[4] = {0.f, 0.f, 0.f, 0.f}, lb[4] = {0.f, 0.f, 0.f, 0.f};      // independent partial sums
+                uint32_t pk[TILE / 64][16];       // bf16 pairs: [2k] = row r0, [2k+1] = row r1, tokens 8k + 2*(lane%4) + {0,1}
+#pragma unroll
+                for (int h = 0; h < TILE / 64; ++h) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        // 2^(s * scale * log2 e - reference): one multiply-add into the exponential unit
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(s[h][4 * k + 0]), scale_log2, ms0));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(s[h][4 * k + 1]), scale_log2, ms0));
+                        const float p2 = ex2_approx(fmaf(__uint_as_float(s[h][4 * k + 2]), scale_log2, ms1));
+                        const float p3 = ex2_approx(fmaf(__uint_as_float(s[h][4 * k + 3]), scale_log2, ms1));
+                        la[k & 3] += p0 + p1; lb[k & 3] += p2 + p3;
+                        pk[h][2 * k] = pack_bf16x2(p0, p1);
+                        pk[h][2 * k + 1] = pack_bf16x2(p2, p3);
+                    }
+                }
+                const float ls0 = (la[0] + la[1]) + (la[2] + la[3]), ls1 = (lb[0] + lb[1]) + (lb[2] + lb[3]);
+                // P and O belong to the tensor core until P V of tile t-1 is done; P V of tile t cannot
+                // start before this warp has published P below.
+                if (t >= 1 && !mbar_wait_warp(&pv_done_bar[(tau - 1) & 1], ((uint32_t)((tau - 1) >> 1)) & 1u, abort_ptr)) { ok = false; break; }
+                if (__any_sync(0xffffffffu, grow)) {
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c0 = 0; c0 < D; c0 += 64) {
+                        uint32_t o[32];
+                        tmem_ld_16x64(tmem_o + lane_base + (uint32_t)c0, o);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            o[4 * k + 0] = __float_as_uint(__uint_as_float(o[4 * k + 0]) * f0);
+                            o[4 * k + 1] = __float_as_uint(__uint_as_float(o[4 * k + 1]) * f0);
+                            o[4 * k + 2] = __float_as_uint(__uint_as_float(o[4 * k + 2]) * f1);
+                            o[4 * k + 3] = __float_as_uint(__uint_as_float(o[4 * k + 3]) * f1);
+                        }
+                        tmem_st_16x64(tmem_o + lane_base + (uint32_t)c0, o);
+                    }
+                    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                    l_run[0] *= f0; l_run[1] *= f1;
+                }
+#pragma unroll
+                for (int h = 0; h < TILE / 64; ++h) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        // tokens 8k .. 8k+7 of the 64-token group are 16-byte unit k of the row
+                        // (r1 = r0 + 8 has the same swizzle phase: row & 7)
+                        *reinterpret_cast<uint32_t*>(p_row0 + h * Cfg::kQRegion + ((k ^ (r0 & 7)) << 4)) = pk[h][2 * k];
+                        *reinterpret_cast<uint32_t*>(p_row0 + h * Cfg::kQRegion + 8 * 128 + ((k ^ (r0 & 7)) << 4)) = pk[h][2 * k + 1];
+                    }
+                }
+                l_run[0] += ls0; l_run[1] += ls1;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // P is read by the tensor core
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_full_bar[buf]);
+            }
+            const int tau_last = tau_base + n_tiles - 1;
+            if (ok && !mbar_wait_warp(&pv_done_bar[tau_last & 1], ((uint32_t)(tau_last >> 1)) & 1u, abort_ptr)) ok = false;
+            tc_fence_after();
+            tau_base += n_tiles;
+            if (!ok) break;
+            // ---- this piece's result: normalised output if it is the whole pair, else (O, max, sum)
             l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 1);
             l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], 2);
             l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
             l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
-            const bool single = n_chunks_b == 1;
-            const int rows_pad = (rows + 15) / 16 * 16;
-            const size_t item = ((size_t)b * p.Hkv + g) * p.max_chunks + chunk;
+            const bool single = sg.part_o == nullptr;
             const float inv0 = 1.f / l_run[0], inv1 = 1.f / l_run[1];
             const size_t out0 = r0 < rows ? (((size_t)b * p.R + r0 / G) * p.Hq + g * G + r0 % G) : 0;
             const size_t out1 = r1 < rows ? (((size_t)b * p.R + r1 / G) * p.Hq + g * G + r1 % G) : 0;
@@ -417,8 +617,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                             if (p.out_f32) *reinterpret_cast<float2*>(p.out_f32 + out1 * D + c) = make_float2(a2, a3);
                         }
                     } else {
-                        if (r0 < rows) *reinterpret_cast<float2*>(p.part_o + (item * rows_pad + r0) * D + c) = make_float2(a0, a1);
-                        if (r1 < rows) *reinterpret_cast<float2*>(p.part_o + (item * rows_pad + r1) * D + c) = make_float2(a2, a3);
+                        if (r0 < rows) *reinterpret_cast<float2*>(sg.part_o + (size_t)r0 * D + c) = make_float2(a0, a1);
+                        if (r1 < rows) *reinterpret_cast<float2*>(sg.part_o + (size_t)r1 * D + c) = make_float2(a2, a3);
                     }
                 }
             }
@@ -429,13 +629,14 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                         if (r1 < rows) p.lse[out1] = (m_ref[1] + log2f(l_run[1])) * 0.6931471805599453f;
                     }
                 } else {
-                    if (r0 < rows) { p.part_ml[(item * rows_pad + r0) * 2] = m_ref[0]; p.part_ml[(item * rows_pad + r0) * 2 + 1] = l_run[0]; }
-                    if (r1 < rows) { p.part_ml[(item * rows_pad + r1) * 2] = m_ref[1]; p.part_ml[(item * rows_pad + r1) * 2 + 1] = l_run[1]; }
+                    if (r0 < rows) { sg.part_ml[r0 * 2] = m_ref[0]; sg.part_ml[r0 * 2 + 1] = l_run[0]; }
+                    if (r1 < rows) { sg.part_ml[r1 * 2] = m_ref[1]; sg.part_ml[r1 * 2 + 1] = l_run[1]; }
                 }
             }
         }
     }
 
+    pdl_trigger();
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -446,14 +647,80 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
 }
 
+// Merge the pieces of every (sequence, KV head) pair that the flat schedule cut: one CTA per
+// (sequence, KV head, query row), one thread per channel.  The pieces of a pair sit in consecutive
+// CTAs of the split kernel; piece c is in slot 0 of CTA c unless the pair begins inside that CTA's range.
+__global__ void __launch_bounds__(128) attn_flat_combine_kernel(const AttnParams p, int rows_pad) {
+    const int G = p.Hq / p.Hkv, rows = G * p.R;
+    const int r = blockIdx.x % rows, g = (blockIdx.x / rows) % p.Hkv, b = blockIdx.x / (rows * p.Hkv);
+    pdl_wait();
+    pdl_trigger();
+    const int per_cta = p.flat_meta[0];
+    const int n_b = p.flat_meta[2 + b + 1] - p.flat_meta[2 + b];
+    if (n_b <= 0) return;
+    const int start = p.flat_meta[2 + b] * p.Hkv + g * n_b, end = start + n_b;
+    const int c_first = start / per_cta, c_last = (end - 1) / per_cta;
+    if (c_first == c_last) return;                 // the pair was finished by one CTA
+    __shared__ float s_w[kFlatMaxCtas];            // first the piece maxima, then the merge weights
+    __shared__ float s_l[kFlatMaxCtas];
+    const int n = c_last - c_first + 1;
+    auto slot_of = [&](int i) -> size_t { const int c = c_first + i; return (size_t)c * 2 + (start <= c * per_cta ? 0 : 1); };
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const float2 ml = *reinterpret_cast<const float2*>(p.flat_part_ml + (slot_of(i) * rows_pad + r) * 2);
+        s_w[i] = ml.x;
+        s_l[i] = ml.y;
+    }
+    __syncthreads();
+    float M = -INFINITY;
+    for (int i = 0; i < n; ++i) M = fmaxf(M, s_w[i]);
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) s_w[i] = s_w[i] == -INFINITY ? 0.f : exp2f(s_w[i] - M);
+    __syncthreads();
+    float Lsum = 0.f;
+    for (int i = 0; i < n; ++i) Lsum += s_l[i] * s_w[i];
+    const float inv = 1.f / Lsum;
+    const size_t row_out = ((size_t)b * p.R + r / G) * p.Hq + g * G + r % G;
+    for (int col = threadIdx.x; col < p.d; col += blockDim.x) {
+        float acc = 0.f;
+        for (int i = 0; i < n; ++i) acc += p.flat_part_o[(slot_of(i) * rows_pad + r) * p.d + col] * s_w[i];      // piece order
+        acc *= inv;
+        p.out[row_out * p.d + col] = __float2bfloat16(acc);
+        if (p.out_f32) p.out_f32[row_out * p.d + col] = acc;
+    }
+    if (p.lse && threadIdx.x == 0) p.lse[row_out] = (M + log2f(Lsum)) * 0.6931471805599453f;
+}
+
+int flat_sm_count() {
+    static int n = 0;
+    if (n) return n;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        n = 148;
+    return n;
+}
+
 template <int D, int TILE>
-cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream) {
+cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream, bool flat, int* launched) {
     using Cfg = UmmaAttnCfg<D, TILE>;
     static_assert(Cfg::kColsNeeded <= 512, "S buffers and O fit tensor memory");
     static_assert(Cfg::kSmem <= 227 * 1024, "ring, Q and P fit shared memory");
-    cudaError_t e = cudaFuncSetAttribute(attn_umma_kernel<D, TILE>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
+    cudaError_t e;
+    if (flat) {
+        e = cudaFuncSetAttribute(attn_umma_kernel<D, TILE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
+        if (e != cudaSuccess) return e;
+        int ctas = flat_sm_count() * Cfg::kCtasPerSm;
+        if (ctas > kFlatMaxCtas) ctas = kFlatMaxCtas;
+        e = launch_pdl(attn_umma_kernel<D, TILE, true>, dim3(ctas), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, p);
+        if (e != cudaSuccess) return e;
+        const int rows = (p.Hq / p.Hkv) * p.R;
+        e = launch_pdl(attn_flat_combine_kernel, dim3(p.B * p.Hkv * rows), dim3(p.d < 128 ? 64 : 128), 0, stream, p, attn_rows_pad(rows));
+        *launched = 2;
+        return e;
+    }
+    e = cudaFuncSetAttribute(attn_umma_kernel<D, TILE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
     if (e != cudaSuccess) return e;
-    return launch_pdl(attn_umma_kernel<D, TILE>, dim3(p.max_chunks, p.Hkv, p.B), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, p);
+    *launched = 1;
+    return launch_pdl(attn_umma_kernel<D, TILE, false>, dim3(p.max_chunks, p.Hkv, p.B), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, p);
 }
 
 }  // namespace
@@ -463,11 +730,16 @@ bool attn_umma_supported(const AttnParams& p) {
            p.kv_chunk <= kUmmaMaxChunkPages * kPageSize && p.kv_chunk % 64 == 0;
 }
 
-cudaError_t launch_attn_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream) {
+// The flat schedule needs the batch's tile counts in shared memory.
+bool attn_umma_flat_supported(const AttnParams& p) { return attn_umma_supported(p) && p.B <= kFlatMaxBatch; }
+
+// *launched: kernels launched; *needs_chunk_combine: the chunk merge kernel still has to run.
+cudaError_t launch_attn_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream, bool flat,
+                             int* launched) {
     switch (p.d) {
-        case 64: return launch_umma<64, 64>(p, mk, mv, stream);
-        case 128: return launch_umma<128, 64>(p, mk, mv, stream);
-        case 256: return launch_umma<256, 64>(p, mk, mv, stream);
+        case 64: return launch_umma<64, 64>(p, mk, mv, stream, flat, launched);
+        case 128: return launch_umma<128, 64>(p, mk, mv, stream, flat, launched);
+        case 256: return launch_umma<256, 64>(p, mk, mv, stream, flat, launched);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -24,13 +24,24 @@ struct AttnParams {
     float* part_ml;    // [B, Hkv, max_chunks, rows_pad, 2] running max (log2 domain) and sum
     int32_t* dev_status;
     int path;          // 0: choose by shape, 1: warp-level MMA kernel, 2: tcgen05 kernel
+    bool chunk_forced; // the caller fixed kv_chunk: keep the (chunk, KV head, sequence) grid
+    // flat schedule of the tcgen05 kernel: two partial slots per resident CTA, and what the merge needs
+    float* flat_part_o;    // [kFlatMaxCtas * 2, rows_pad, d]
+    float* flat_part_ml;   // [kFlatMaxCtas * 2, rows_pad, 2]
+    int32_t* flat_meta;    // [0] tiles per CTA, [1] tiles in all, [2 + b] tiles of sequences 0 .. b-1 (per KV head)
 };
+constexpr int kFlatMaxCtas = 320;      // resident CTAs of the flat schedule (two per SM)
+constexpr int kFlatMaxBatchMeta = 1024;
 int attn_rows_pad(int group_rows);                 // query rows per KV head, padded to the MMA tile
 cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream);
 // tcgen05 variant of the split kernel (attn_umma.cu); the tensor maps are the ones the warp-MMA kernel uses
 bool attn_umma_supported(const AttnParams& p);
+bool attn_umma_flat_supported(const AttnParams& p);
 bool attn_use_umma(const AttnParams& p);
-cudaError_t launch_attn_umma(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream);
+// flat: balanced persistent schedule with its own merge kernel; otherwise the chunk grid, merged by the caller.
+// *launched receives the number of kernels launched.
+cudaError_t launch_attn_umma(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream, bool flat,
+                             int* launched);
 
 // ---------------------------------------------------------------- LM head
 struct LmHeadParams {
