@@ -457,11 +457,13 @@ int attn_rows_pad(int group_rows) { return (group_rows + 15) / 16 * 16; }
 
 // Which split kernel runs.  The warp-MMA kernel re-reads every K/V tile from shared memory once
 // per 16 query rows, which saturates the shared-memory pipe from about 48 rows up; the tcgen05
-// kernel reads each tile once whatever the row count.
+// kernel reads each tile once whatever the row count, and with its balanced schedule it is the
+// faster one on every head_dim <= 128 shape measured.  At head_dim 256 its ring leaves room for one
+// CTA per SM only, and the warp-MMA kernel (few rows per KV head on such models) stays ahead.
 bool attn_use_umma(const AttnParams& p) {
     if (p.path == 1 || !attn_umma_supported(p)) return false;
     if (p.path == 2) return true;
-    return attn_rows_pad((p.Hq / p.Hkv) * p.R) >= 48;
+    return p.d <= 128;
 }
 
 cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {

@@ -647,47 +647,75 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
 }
 
-// Merge the pieces of every (sequence, KV head) pair that the flat schedule cut: one CTA per
-// (sequence, KV head, query row), one thread per channel.  The pieces of a pair sit in consecutive
-// CTAs of the split kernel; piece c is in slot 0 of CTA c unless the pair begins inside that CTA's range.
-__global__ void __launch_bounds__(128) attn_flat_combine_kernel(const AttnParams p, int rows_pad) {
-    const int G = p.Hq / p.Hkv, rows = G * p.R;
-    const int r = blockIdx.x % rows, g = (blockIdx.x / rows) % p.Hkv, b = blockIdx.x / (rows * p.Hkv);
+// Merge the pieces of every (sequence, KV head) pair that the flat schedule cut: one CTA per pair,
+// all of its query rows.  The pieces of a pair sit in consecutive CTAs of the split kernel; piece c is
+// in slot 0 of CTA c unless the pair begins inside that CTA's range.  Pieces are summed in order.
+constexpr int kFlatCombineThreads = 256;
+__global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(const AttnParams p, int rows_pad, int rows_per_cta) {
+    const int G = p.Hq / p.Hkv;
+    const int g = blockIdx.x % p.Hkv, b = blockIdx.x / p.Hkv;
+    // with few pairs each pair's rows are dealt to several CTAs (blockIdx.y)
+    const int row0 = blockIdx.y * rows_per_cta, rows = min(rows_per_cta, G * p.R - row0);
     pdl_wait();
     pdl_trigger();
     const int per_cta = p.flat_meta[0];
-    const int n_b = p.flat_meta[2 + b + 1] - p.flat_meta[2 + b];
+    const int cum_b = p.flat_meta[2 + b], n_b = p.flat_meta[2 + b + 1] - cum_b;
     if (n_b <= 0) return;
-    const int start = p.flat_meta[2 + b] * p.Hkv + g * n_b, end = start + n_b;
+    const int start = cum_b * p.Hkv + g * n_b, end = start + n_b;
     const int c_first = start / per_cta, c_last = (end - 1) / per_cta;
     if (c_first == c_last) return;                 // the pair was finished by one CTA
-    __shared__ float s_w[kFlatMaxCtas];            // first the piece maxima, then the merge weights
-    __shared__ float s_l[kFlatMaxCtas];
     const int n = c_last - c_first + 1;
     auto slot_of = [&](int i) -> size_t { const int c = c_first + i; return (size_t)c * 2 + (start <= c * per_cta ? 0 : 1); };
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const float2 ml = *reinterpret_cast<const float2*>(p.flat_part_ml + (slot_of(i) * rows_pad + r) * 2);
-        s_w[i] = ml.x;
-        s_l[i] = ml.y;
+    // per row: the common maximum and 1 / sum; per (piece, row): the merge weight
+    extern __shared__ float s_comb[];
+    float* s_w = s_comb;                           // [n][rows]
+    float* s_inv = s_comb + (size_t)n * rows;      // [rows]
+    for (int rr = threadIdx.x; rr < rows; rr += blockDim.x) {
+        const int r = row0 + rr;
+        float M = -INFINITY;
+        for (int i = 0; i < n; ++i) M = fmaxf(M, p.flat_part_ml[(slot_of(i) * rows_pad + r) * 2]);
+        float Lsum = 0.f;
+        for (int i = 0; i < n; ++i) {
+            const float2 ml = *reinterpret_cast<const float2*>(p.flat_part_ml + (slot_of(i) * rows_pad + r) * 2);
+            const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+            s_w[(size_t)i * rows + rr] = w;
+            Lsum += ml.y * w;
+        }
+        s_inv[rr] = 1.f / Lsum;
+        if (p.lse) p.lse[((size_t)b * p.R + r / G) * p.Hq + g * G + r % G] = (M + log2f(Lsum)) * 0.6931471805599453f;
     }
     __syncthreads();
-    float M = -INFINITY;
-    for (int i = 0; i < n; ++i) M = fmaxf(M, s_w[i]);
-    __syncthreads();
-    for (int i = threadIdx.x; i < n; i += blockDim.x) s_w[i] = s_w[i] == -INFINITY ? 0.f : exp2f(s_w[i] - M);
-    __syncthreads();
-    float Lsum = 0.f;
-    for (int i = 0; i < n; ++i) Lsum += s_l[i] * s_w[i];
-    const float inv = 1.f / Lsum;
-    const size_t row_out = ((size_t)b * p.R + r / G) * p.Hq + g * G + r % G;
-    for (int col = threadIdx.x; col < p.d; col += blockDim.x) {
-        float acc = 0.f;
-        for (int i = 0; i < n; ++i) acc += p.flat_part_o[(slot_of(i) * rows_pad + r) * p.d + col] * s_w[i];      // piece order
-        acc *= inv;
-        p.out[row_out * p.d + col] = __float2bfloat16(acc);
-        if (p.out_f32) p.out_f32[row_out * p.d + col] = acc;
+    const int quads = p.d / 4;                     // a thread produces four channels of one row at a time
+    for (int idx = threadIdx.x; idx < rows * quads; idx += blockDim.x) {
+        const int rr = idx / quads, r = row0 + rr, c = (idx % quads) * 4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        int i = 0;
+        for (; i + 4 <= n; i += 4) {                // four independent loads in flight, summed in piece order
+            const float4 v0 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i) * rows_pad + r) * p.d + c);
+            const float4 v1 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i + 1) * rows_pad + r) * p.d + c);
+            const float4 v2 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i + 2) * rows_pad + r) * p.d + c);
+            const float4 v3 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i + 3) * rows_pad + r) * p.d + c);
+            const float w0 = s_w[(size_t)i * rows + rr], w1 = s_w[(size_t)(i + 1) * rows + rr];
+            const float w2 = s_w[(size_t)(i + 2) * rows + rr], w3 = s_w[(size_t)(i + 3) * rows + rr];
+            acc.x += v0.x * w0; acc.y += v0.y * w0; acc.z += v0.z * w0; acc.w += v0.w * w0;
+            acc.x += v1.x * w1; acc.y += v1.y * w1; acc.z += v1.z * w1; acc.w += v1.w * w1;
+            acc.x += v2.x * w2; acc.y += v2.y * w2; acc.z += v2.z * w2; acc.w += v2.w * w2;
+            acc.x += v3.x * w3; acc.y += v3.y * w3; acc.z += v3.z * w3; acc.w += v3.w * w3;
+        }
+        for (; i < n; ++i) {
+            const float4 v = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i) * rows_pad + r) * p.d + c);
+            const float w = s_w[(size_t)i * rows + rr];
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
+        const float inv = s_inv[rr];
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        const size_t row_out = ((size_t)b * p.R + r / G) * p.Hq + g * G + r % G;
+        uint2 packed;
+        packed.x = pack_bf16x2(acc.x, acc.y);
+        packed.y = pack_bf16x2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(p.out + row_out * p.d + c) = packed;
+        if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row_out * p.d + c) = acc;
     }
-    if (p.lse && threadIdx.x == 0) p.lse[row_out] = (M + log2f(Lsum)) * 0.6931471805599453f;
 }
 
 int flat_sm_count() {
@@ -713,7 +741,18 @@ cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtens
         e = launch_pdl(attn_umma_kernel<D, TILE, true>, dim3(ctas), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, p);
         if (e != cudaSuccess) return e;
         const int rows = (p.Hq / p.Hkv) * p.R;
-        e = launch_pdl(attn_flat_combine_kernel, dim3(p.B * p.Hkv * rows), dim3(p.d < 128 ? 64 : 128), 0, stream, p, attn_rows_pad(rows));
+        // weights for at most `ctas` pieces of a pair (a pair can span every CTA), plus one value per row
+        // enough CTAs to fill the machine: a pair's rows are dealt to several CTAs when there are few pairs
+        const int pairs = p.B * p.Hkv;
+        int row_groups = (2 * flat_sm_count() + pairs - 1) / pairs;
+        if (row_groups > rows) row_groups = rows;
+        const int rows_per_cta = (rows + row_groups - 1) / row_groups;
+        row_groups = (rows + rows_per_cta - 1) / rows_per_cta;
+        const size_t comb_smem = ((size_t)ctas + 1) * rows_per_cta * sizeof(float);
+        e = cudaFuncSetAttribute(attn_flat_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)comb_smem);
+        if (e != cudaSuccess) return e;
+        const int threads = rows_per_cta * (p.d / 4) <= 64 ? 64 : (rows_per_cta * (p.d / 4) <= 128 ? 128 : kFlatCombineThreads);
+        e = launch_pdl(attn_flat_combine_kernel, dim3(pairs, row_groups), dim3(threads), comb_smem, stream, p, attn_rows_pad(rows), rows_per_cta);
         *launched = 2;
         return e;
     }
