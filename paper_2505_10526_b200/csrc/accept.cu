@@ -19,6 +19,7 @@ constexpr int kScanThreads = 256;
 constexpr int kScanBatch = 6;     // partial slots a lane loads before merging (192 slots = one batch)
 constexpr int kSampleThreads = 256;
 constexpr int kPerThread = kResidualChunk / kSampleThreads;   // 16 contiguous entries per thread
+constexpr int kWalkChunks = 512;  // chunk masses staged in shared memory for the walk (vocabularies up to 2M entries)
 static_assert(kPerThread == 16, "chunk layout");
 
 struct Stat {
@@ -209,17 +210,24 @@ __global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptP
     if (!s_flag) return;
     __threadfence();
 
+    // The walk over the chunk masses is sequential (fixed summation order) but its loads need not be:
+    // the CTA fetches the masses the other CTAs wrote (L2, bypassing L1) into shared memory at once.
+    __shared__ double s_sums[kWalkChunks];
+    const bool staged = p.n_chunks <= kWalkChunks;
     int use_q = st.use_q;
     for (int attempt = 0; attempt < 2; ++attempt) {
-        // sequential walk over the chunk masses (a few dozen doubles)
+        if (staged) {
+            for (int i = t; i < p.n_chunks; i += kSampleThreads) s_sums[i] = __ldcg(sums + i);
+            __syncthreads();
+        }
         if (t == 0) {
             double tot = 0.0;
-            for (int i = 0; i < p.n_chunks; ++i) tot += ((volatile double*)sums)[i];
+            for (int i = 0; i < p.n_chunks; ++i) tot += staged ? s_sums[i] : ((volatile double*)sums)[i];
             const double target = (double)p.u_sample[(size_t)b * R + st.n] * tot;
             int pick = -1, last_pos = -1;
             double cum = 0.0, base = 0.0;
             for (int i = 0; i < p.n_chunks; ++i) {
-                const double s = ((volatile double*)sums)[i];
+                const double s = staged ? s_sums[i] : ((volatile double*)sums)[i];
                 if (s > 0.0) last_pos = i;
                 if (pick < 0 && s > 0.0 && cum + s > target) { pick = i; base = cum; }
                 cum += s;
@@ -242,6 +250,7 @@ __global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptP
             block_exclusive_scan(loc, warp_sums, &tt);
             if (t == 0) sums[cc] = tt;
         }
+        __threadfence();       // this CTA reads the new masses back through L2 on the second attempt
         __syncthreads();
     }
     const int pick = s_pick[0];

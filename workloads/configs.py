@@ -95,6 +95,12 @@ for _g in (5, 7):
     _add(replace(CONFIGS[f"qwen7b_long_g{_g}_t0"], name=f"qwen7b_long_b16_g{_g}_t0", batch=16))
 
 
+# The LM-head shapes of the long-context sweep (M = 256 / 384 / 512 rows) with short contexts: the
+# acceptance call is the same, the attention part is small enough for multi-pass profiler captures.
+for _g in (3, 5, 7):
+    _add(replace(CONFIGS[f"qwen7b_long_g{_g}_t0"], name=f"qwen7b_lmhead_g{_g}_t0", ctx_lo=64, ctx_hi=256, image_tokens=0.25))
+
+
 def get_config(name: str) -> VerifyConfig:
     if name not in CONFIGS:
         raise KeyError(f"unknown workload {name!r}; known: {sorted(CONFIGS)}")
