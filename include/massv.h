@@ -251,6 +251,20 @@ int massv_version(void);
  * (diagnostic; lets a caller confirm that a call really ran on the device). */
 uint64_t massv_launch_count(void);
 
+/*
+ * Measurement hook (no counterpart in the paper).  massv_accept and massv_verify_attn launch several
+ * kernels each; a caller that wants the duration of the dominant one alone (the LM-head GEMM, the
+ * attention split kernel) hands in two CUDA events per call, and the library records `start`
+ * immediately before and `stop` immediately after that kernel on the call's stream.  The setting is
+ * per host thread and stays until changed; NULL for both switches a hook off.  Events are
+ * cudaEvent_t handles created with timing enabled and owned by the caller.  Recording them keeps
+ * the timed kernel from overlapping with its neighbours in the stream, so leave the hooks off on
+ * calls whose end-to-end time matters.
+ */
+typedef struct CUevent_st *massv_event_t;     /* a cudaEvent_t */
+int massv_set_timing_events(massv_event_t lm_head_start, massv_event_t lm_head_stop,
+                            massv_event_t attn_start, massv_event_t attn_stop);
+
 #ifdef __cplusplus
 }
 #endif

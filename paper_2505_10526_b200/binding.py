@@ -64,6 +64,8 @@ def _load():
     lib.massv_strerror.argtypes = [ctypes.c_int]
     lib.massv_version.restype = ctypes.c_int
     lib.massv_launch_count.restype = ctypes.c_uint64
+    lib.massv_set_timing_events.restype = ctypes.c_int
+    lib.massv_set_timing_events.argtypes = [vp, vp, vp, vp]
     return lib
 
 
@@ -96,6 +98,21 @@ def massv_version() -> int:
 
 def massv_launch_count() -> int:
     return int(_lib.massv_launch_count())
+
+
+def massv_set_timing_events(lm_head=None, attn=None) -> None:
+    """Record pairs of torch CUDA events (created with enable_timing=True) around the LM-head kernel
+    and / or the attention split kernel of the following calls on this thread; None switches a hook off."""
+    def handles(pair):
+        if pair is None:
+            return None, None
+        for ev in pair:
+            if not getattr(ev, "cuda_event", 0):
+                ev.record()                 # torch creates the underlying CUDA event lazily
+        return ctypes.c_void_p(pair[0].cuda_event), ctypes.c_void_p(pair[1].cuda_event)
+    rc = _lib.massv_set_timing_events(*handles(lm_head), *handles(attn))
+    if rc != 0:
+        raise MassvError(rc, "massv_set_timing_events")
 
 
 def massv_strerror(status: int) -> str:

@@ -11,6 +11,10 @@ using namespace massv;
 static std::atomic<uint64_t> g_launches{0};
 namespace massv {
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+TimingHooks& timing_hooks() {
+    static thread_local TimingHooks hooks;
+    return hooks;
+}
 }
 
 namespace {
@@ -261,6 +265,18 @@ const char* massv_strerror(int status) {
 }
 
 int massv_version(void) { return 100; }
+
+int massv_set_timing_events(massv_event_t lm_head_start, massv_event_t lm_head_stop, massv_event_t attn_start,
+                            massv_event_t attn_stop) {
+    if ((lm_head_start == nullptr) != (lm_head_stop == nullptr) || (attn_start == nullptr) != (attn_stop == nullptr))
+        return MASSV_ERR_INVALID_ARG;
+    TimingHooks& h = timing_hooks();
+    h.lm_head_start = reinterpret_cast<cudaEvent_t>(lm_head_start);
+    h.lm_head_stop = reinterpret_cast<cudaEvent_t>(lm_head_stop);
+    h.attn_start = reinterpret_cast<cudaEvent_t>(attn_start);
+    h.attn_stop = reinterpret_cast<cudaEvent_t>(attn_stop);
+    return MASSV_OK;
+}
 
 uint64_t massv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -476,10 +476,12 @@ cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
     const int rows = (p.Hq / p.Hkv) * p.R;
     const int mt = attn_rows_pad(rows) / 16;
     cudaError_t e;
+    const TimingHooks& hooks = timing_hooks();
+    if (hooks.attn_start && cudaEventRecord(hooks.attn_start, stream) != cudaSuccess) return cudaGetLastError();
     if (attn_use_umma(p)) {
         const bool flat = !p.chunk_forced && attn_umma_flat_supported(p);
         int launched = 0;
-        e = launch_attn_umma(p, mk, mv, stream, flat, &launched);
+        e = launch_attn_umma(p, mk, mv, stream, flat, &launched, hooks.attn_stop);
         if (e != cudaSuccess) return e;
         if (flat) {
             count_launches(launched);
@@ -494,6 +496,7 @@ cudaError_t launch_verify_attn(const AttnParams& p, cudaStream_t stream) {
         }
     }
     if (e != cudaSuccess) return e;
+    if (hooks.attn_stop && cudaEventRecord(hooks.attn_stop, stream) != cudaSuccess) return cudaGetLastError();
     int launched = 1;
     if (p.max_chunks > 1) {
         if (p.max_chunks > kCombineMaxChunks) return cudaErrorInvalidValue;

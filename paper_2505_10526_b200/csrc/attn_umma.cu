@@ -728,7 +728,8 @@ int flat_sm_count() {
 }
 
 template <int D, int TILE>
-cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream, bool flat, int* launched) {
+cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream, bool flat, int* launched,
+                        cudaEvent_t split_done) {
     using Cfg = UmmaAttnCfg<D, TILE>;
     static_assert(Cfg::kColsNeeded <= 512, "S buffers and O fit tensor memory");
     static_assert(Cfg::kSmem <= 227 * 1024, "ring, Q and P fit shared memory");
@@ -740,6 +741,7 @@ cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtens
         if (ctas > kFlatMaxCtas) ctas = kFlatMaxCtas;
         e = launch_pdl(attn_umma_kernel<D, TILE, true>, dim3(ctas), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, p);
         if (e != cudaSuccess) return e;
+        if (split_done && cudaEventRecord(split_done, stream) != cudaSuccess) return cudaGetLastError();
         const int rows = (p.Hq / p.Hkv) * p.R;
         // weights for at most `ctas` pieces of a pair (a pair can span every CTA), plus one value per row
         // enough CTAs to fill the machine: a pair's rows are dealt to several CTAs when there are few pairs
@@ -774,11 +776,11 @@ bool attn_umma_flat_supported(const AttnParams& p) { return attn_umma_supported(
 
 // *launched: kernels launched; *needs_chunk_combine: the chunk merge kernel still has to run.
 cudaError_t launch_attn_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream, bool flat,
-                             int* launched) {
+                             int* launched, cudaEvent_t split_done) {
     switch (p.d) {
-        case 64: return launch_umma<64, 64>(p, mk, mv, stream, flat, launched);
-        case 128: return launch_umma<128, 64>(p, mk, mv, stream, flat, launched);
-        case 256: return launch_umma<256, 64>(p, mk, mv, stream, flat, launched);
+        case 64: return launch_umma<64, 64>(p, mk, mv, stream, flat, launched, split_done);
+        case 128: return launch_umma<128, 64>(p, mk, mv, stream, flat, launched, split_done);
+        case 256: return launch_umma<256, 64>(p, mk, mv, stream, flat, launched, split_done);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -75,6 +75,12 @@ struct SeqState {
     float inv_sum;    // 1 / sum exp((z - max)/T) of row n
 };
 
+// Optional per-thread timing hooks (massv_set_timing_events): events recorded around the dominant kernel of a call.
+struct TimingHooks {
+    cudaEvent_t lm_head_start = nullptr, lm_head_stop = nullptr, attn_start = nullptr, attn_stop = nullptr;
+};
+TimingHooks& timing_hooks();
+
 // Host-side tally of kernel launches (see massv_launch_count).
 void count_launches(int n);
 

@@ -40,8 +40,9 @@ bool attn_umma_flat_supported(const AttnParams& p);
 bool attn_use_umma(const AttnParams& p);
 // flat: balanced persistent schedule with its own merge kernel; otherwise the chunk grid, merged by the caller.
 // *launched receives the number of kernels launched.
+// split_done, when not null, is recorded right after the split kernel (before any merge kernel).
 cudaError_t launch_attn_umma(const AttnParams& p, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream, bool flat,
-                             int* launched);
+                             int* launched, cudaEvent_t split_done);
 
 // ---------------------------------------------------------------- LM head
 struct LmHeadParams {

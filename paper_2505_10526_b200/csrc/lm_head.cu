@@ -539,6 +539,8 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
 
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     cudaError_t e;
+    const TimingHooks& hooks = timing_hooks();
+    if (hooks.lm_head_start && cudaEventRecord(hooks.lm_head_start, stream) != cudaSuccess) return cudaGetLastError();
     if (pair) {
         e = cudaFuncSetAttribute(lm_head_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -551,6 +553,7 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
                        map_w[1], map_w[2], map_w[3], map_w[4], map_h, p);
     }
     if (e != cudaSuccess) return e;
+    if (hooks.lm_head_stop && cudaEventRecord(hooks.lm_head_stop, stream) != cudaSuccess) return cudaGetLastError();
     count_launches(1);
     return cudaGetLastError();
 }

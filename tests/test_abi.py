@@ -89,3 +89,14 @@ def test_binding_refuses_cpu_tensors(mv):
     x = torch.zeros(8, dtype=torch.bfloat16)
     with pytest.raises(ValueError):
         mv.massv_accept(d, x, x, None, None, None, None, None, None)
+
+
+def test_timing_hook_rejects_half_a_pair(mv):
+    """massv_set_timing_events takes events in pairs; one without the other is refused (host-only check)."""
+    lib = ctypes.CDLL(mv.LIB_PATH)
+    lib.massv_set_timing_events.restype = ctypes.c_int
+    lib.massv_set_timing_events.argtypes = [ctypes.c_void_p] * 4
+    assert lib.massv_set_timing_events(None, None, None, None) == 0
+    assert lib.massv_set_timing_events(ctypes.c_void_p(8), None, None, None) == -1
+    assert lib.massv_set_timing_events(None, None, None, ctypes.c_void_p(8)) == -1
+    assert lib.massv_set_timing_events(None, None, None, None) == 0

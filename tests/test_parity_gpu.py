@@ -352,3 +352,31 @@ def test_gamma_zero_sampling_is_the_draft_side_step():
     for b in range(cfg.batch):
         if ref["margin_sample"][b] >= 1e-3:
             assert toks[b] == int(np.searchsorted(cdf[b], u[b] * cdf[b, -1], side="right"))
+
+
+def test_timing_hook_brackets_the_dominant_kernels():
+    """Events handed to massv_set_timing_events are recorded around the LM-head kernel and the attention
+    split kernel: both intervals are positive and lie inside the interval of the whole step; with the hook
+    switched off again the events are not touched."""
+    import paper_2505_10526_b200 as mv
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = get_config("qwen7b_b1_t0")
+    w = generate(cfg, device="cuda")
+    step = VerifyStep.for_workload(cfg, w)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+    step.run(w, commit=False)                       # warm-up
+    try:
+        ev[0].record()
+        mv.massv_set_timing_events(lm_head=(ev[1], ev[2]), attn=(ev[3], ev[4]))
+        step.run(w, commit=False)
+    finally:
+        mv.massv_set_timing_events(None, None)
+    ev[5].record()
+    torch.cuda.synchronize()
+    whole, lm, attn = ev[0].elapsed_time(ev[5]), ev[1].elapsed_time(ev[2]), ev[3].elapsed_time(ev[4])
+    assert 0.0 < attn < whole and 0.0 < lm < whole
+    assert ev[0].elapsed_time(ev[3]) >= 0.0 and ev[4].elapsed_time(ev[1]) >= 0.0 and ev[2].elapsed_time(ev[5]) >= 0.0
+    assert lm > 0.1          # 1.09 GB of weights cannot be read in less than 0.1 ms
+    step.run(w, commit=False)
+    torch.cuda.synchronize()
+    assert ev[1].elapsed_time(ev[2]) == lm          # not re-recorded once the hook is off
