@@ -380,3 +380,47 @@ def test_timing_hook_brackets_the_dominant_kernels():
     step.run(w, commit=False)
     torch.cuda.synchronize()
     assert ev[1].elapsed_time(ev[2]) == lm          # not re-recorded once the hook is off
+
+
+def _attention_only_case(cfg, kernel, kv_chunk=0):
+    """massv_verify_attn alone (no LM head) against the oracle's attention, for shapes whose
+    acceptance part would be out of range or beside the point."""
+    from paper_2505_10526_b200 import VerifyStep
+    w = generate(cfg, device="cuda")
+    before = {k: w[k].clone() for k in ("k_pages", "v_pages", "seq_lens")}
+    step = VerifyStep.for_workload(cfg, w, want_attn_f32=True, attn_kernel=kernel, kv_chunk=kv_chunk)
+    step.attn(w)
+    torch.cuda.synchronize()
+    assert int(step.dev_status.item()) == 0
+    # the oracle appends the block to copies of the pools as they were before the call, then attends
+    kp, vp = oracle.bf16_bits(before["k_pages"]).copy(), oracle.bf16_bits(before["v_pages"]).copy()
+    pt = w["page_table"].cpu().numpy().astype(np.int32)
+    seq = before["seq_lens"].cpu().numpy().astype(np.int32)
+    oracle.kv_append(oracle.bf16_bits(w["k_new"]), oracle.bf16_bits(w["v_new"]), kp, vp, pt, seq)
+    out, lse = oracle.verify_attn(oracle.bf16_bits(w["q"]), kp, vp, pt, seq)
+    ref = dict(attn_out=out, lse=lse, k_pages=kp, v_pages=vp)
+    err = float(np.abs(step.attn_out_f32.cpu().double().numpy() - ref["attn_out"]).max())
+    err16 = float(np.abs(step.attn_out.cpu().double().numpy() - ref["attn_out"]).max())
+    lse_err = float(np.abs(step.lse.cpu().double().numpy() - ref["lse"]).max())
+    _report(dict(config=cfg.name, kernel=kernel, attn_err_f32=err, attn_err_bf16=err16, lse_err=lse_err))
+    assert err < TOL_ATTN_F32 and err16 < TOL_ATTN_BF16 and lse_err < TOL_LSE
+    assert np.array_equal(oracle.bf16_bits(w["k_pages"]), ref["k_pages"]) and np.array_equal(oracle.bf16_bits(w["v_pages"]), ref["v_pages"])
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_one_long_sequence_is_cut_across_many_ctas(kernel):
+    """A single 20,000-token context: with the balanced schedule each (sequence, head) pair is cut
+    into about sixty pieces held by consecutive CTAs, all merged by the second kernel."""
+    from dataclasses import replace
+    cfg = replace(get_config("qwen7b_b1_t0"), name="one_long_sequence", ctx_lo=20000, ctx_hi=20000, hidden=256, vocab=1024, seed=31)
+    _attention_only_case(cfg, kernel)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_batch_beyond_the_balanced_schedule_limit(kernel):
+    """1,100 short sequences: more than the balanced schedule indexes in shared memory, so the
+    tcgen05 kernel runs on the (chunk, head, sequence) grid; lengths start at zero."""
+    from workloads import VerifyConfig
+    cfg = VerifyConfig(name="big_batch", batch=1100, gamma=1, n_q_heads=4, n_kv_heads=2, head_dim=64, hidden=64, vocab=64,
+                       temperature=0.0, ctx_lo=0, ctx_hi=90, image_tokens=0.25, draft_noise_std=0.5, seed=77)
+    _attention_only_case(cfg, kernel)
