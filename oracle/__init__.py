@@ -123,6 +123,21 @@ def tvd(p, q):
     return float(_load().oracle_tvd(p.shape[0], _p(p, np.float64), _p(q, np.float64)))
 
 
+def sample_top_p(z, u, T, top_p, want_q=True):
+    """Nucleus sampling of softmax(z / T), row by row: z f32 [rows, V], u f32 [rows].
+    Returns dict(token, q (f64 [rows, V] or None), nucleus_size, margin_set, margin_sample)."""
+    rows, V = z.shape
+    token = np.zeros((rows,), dtype=np.int32)
+    size = np.zeros((rows,), dtype=np.int32)
+    q = np.zeros((rows, V), dtype=np.float64) if want_q else None
+    m_set = np.zeros((rows,), dtype=np.float64)
+    m_sample = np.zeros((rows,), dtype=np.float64)
+    _load().oracle_sample_top_p(rows, V, ctypes.c_double(T), ctypes.c_double(top_p), _p(z, np.float32), _p(u, np.float32),
+                                _p(token, np.int32), _p(q, np.float64), _p(size, np.int32), _p(m_set, np.float64),
+                                _p(m_sample, np.float64))
+    return dict(token=token, q=q, nucleus_size=size, margin_set=m_set, margin_sample=m_sample)
+
+
 def verify_step(w, temperature, scale=None, want_attention=True, window=0):
     """Whole verify step on a workload dict of torch tensors (see ``workloads.generate``).
 

@@ -296,6 +296,76 @@ double oracle_tvd(int V, const double *p, const double *q)
     return 0.5 * s;
 }
 
+/*
+ * Nucleus (top-p) sampling of softmax(z / T) (Sec. 3.2: the target's responses for self-distillation are
+ * drawn as sample_top-p(p(. | I, X)); the same rule is the drafter's sampling step when it uses top-p).
+ * Per row: order the tokens by probability, largest first (equal probabilities: lower index first); the
+ * nucleus is the shortest prefix of that order whose mass reaches top_p (the whole vocabulary if rounding
+ * keeps the total below top_p); q = p restricted to the nucleus and renormalised; the token is the inverse
+ * CDF of q in vocabulary order at u (first index whose running mass exceeds u * total; zero-mass tokens
+ * are never returned; if rounding pushes the target past the end, the last nucleus token).
+ *   z [rows, V] fp32 logits, u [rows] in [0, 1)
+ *   token [rows], q_out [rows, V] (may be NULL), nucleus_size [rows],
+ *   margin_set [rows]   : distance of top_p from the nearer of the two prefix masses that decide where the
+ *                         prefix stops (the mass before and after its last token),
+ *   margin_sample [rows]: distance of u from the nearer edge of the drawn token's CDF interval.
+ */
+typedef struct { double p; int v; } oracle_pv;
+static int oracle_pv_cmp(const void *a, const void *b)
+{
+    const oracle_pv *x = (const oracle_pv *)a, *y = (const oracle_pv *)b;
+    if (x->p > y->p) return -1;
+    if (x->p < y->p) return 1;
+    return (x->v > y->v) - (x->v < y->v);
+}
+void oracle_sample_top_p(int rows, int V, double T, double top_p, const float *z, const float *u,
+                         int32_t *token, double *q_out, int32_t *nucleus_size, double *margin_set,
+                         double *margin_sample)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int r = 0; r < rows; ++r) {
+        const float *zr = z + (size_t)r * V;
+        oracle_pv *pv = (oracle_pv *)malloc((size_t)V * sizeof(oracle_pv));
+        char *in = (char *)calloc((size_t)V, 1);
+        double m = -INFINITY, s = 0.0;
+        for (int v = 0; v < V; ++v) if ((double)zr[v] > m) m = (double)zr[v];
+        for (int v = 0; v < V; ++v) s += exp(((double)zr[v] - m) / T);
+        for (int v = 0; v < V; ++v) { pv[v].p = exp(((double)zr[v] - m) / T) / s; pv[v].v = v; }
+        qsort(pv, (size_t)V, sizeof(oracle_pv), oracle_pv_cmp);
+        double cum = 0.0, before = 0.0;
+        int k = 0;
+        while (k < V) {                       /* shortest prefix with mass >= top_p */
+            before = cum;
+            cum += pv[k].p;
+            in[pv[k].v] = 1;
+            ++k;
+            if (cum >= top_p) break;
+        }
+        nucleus_size[r] = k;
+        margin_set[r] = fmin(fabs(top_p - before), fabs(cum - top_p));
+        /* restrict, renormalise (in vocabulary order), draw */
+        double total = 0.0;
+        for (int v = 0; v < V; ++v) if (in[v]) total += exp(((double)zr[v] - m) / T) / s;
+        const double target = (double)u[r] * total;
+        double run = 0.0, lo_edge = 0.0, hi_edge = 0.0;
+        int tok = -1, last = -1;
+        for (int v = 0; v < V; ++v) {
+            const double pr = in[v] ? exp(((double)zr[v] - m) / T) / s : 0.0;
+            if (q_out) q_out[(size_t)r * V + v] = pr / total;
+            if (pr > 0.0) {
+                last = v;
+                if (tok < 0 && run + pr > target) { tok = v; lo_edge = run; hi_edge = run + pr; }
+            }
+            run += pr;
+        }
+        if (tok < 0) { tok = last; lo_edge = hi_edge = total; }
+        token[r] = tok;
+        margin_sample[r] = fmin(fabs((double)u[r] - lo_edge / total), fabs(hi_edge / total - (double)u[r]));
+        free(pv);
+        free(in);
+    }
+}
+
 int oracle_num_threads(void)
 {
 #ifdef _OPENMP

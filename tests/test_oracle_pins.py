@@ -576,3 +576,79 @@ def test_tvd_hand_values():
     assert oracle.tvd(a, a.copy()) == 0.0
     assert abs(oracle.tvd(np.array([1.0, 0.0, 0.0]), np.array([0.0, 0.25, 0.75])) - 1.0) < 1e-15
     assert abs(oracle.tvd(a, b) - oracle.tvd(b, a)) < 1e-18
+
+
+# ---------------------------------------------------------------- nucleus (top-p) sampling (Sec. 3.2)
+def _softmax64(z, T):
+    z = z.astype(np.float64) / T
+    e = np.exp(z - z.max(-1, keepdims=True))
+    return e / e.sum(-1, keepdims=True)
+
+
+def test_top_p_hand_worked_example():
+    """p = (0.5, 0.2, 0.2, 0.1), top_p = 0.6: the prefix (0.5, then the first of the two 0.2s) reaches 0.7,
+    so the nucleus is {0, 1} (the tie goes to the lower index) and q = (5/7, 2/7, 0, 0)."""
+    z = np.log(np.array([[0.5, 0.2, 0.2, 0.1]] * 3, dtype=np.float64)).astype(np.float32)
+    u = np.array([0.70, 0.72, 0.0], dtype=np.float32)
+    r = oracle.sample_top_p(z, u, 1.0, 0.6)
+    assert r["nucleus_size"].tolist() == [2, 2, 2]
+    np.testing.assert_allclose(r["q"][0], [5 / 7, 2 / 7, 0, 0], atol=1e-7)
+    assert r["token"].tolist() == [0, 1, 0]          # 5/7 = 0.714: u = 0.70 falls in token 0, u = 0.72 in token 1
+    np.testing.assert_allclose(r["margin_set"], 0.1, atol=1e-6)      # 0.6 is 0.1 from both 0.5 and 0.7
+    # top_p = 0.7 is reached exactly by the same prefix (>=); 0.71 needs the second 0.2 as well
+    assert oracle.sample_top_p(z[:1], u[:1], 1.0, 0.7 - 1e-9)["nucleus_size"][0] == 2
+    assert oracle.sample_top_p(z[:1], u[:1], 1.0, 0.71)["nucleus_size"][0] == 3
+
+
+def test_top_p_against_a_stable_argsort_reference():
+    """Independent formulation with numpy: stable argsort of -p, cumulative sum, cut, renormalise,
+    searchsorted on the vocabulary-order CDF."""
+    rng = np.random.default_rng(5)
+    for V, T, top_p in [(16, 1.0, 0.5), (257, 0.7, 0.9), (1000, 1.3, 0.25), (64, 1.0, 0.999)]:
+        z = (rng.standard_normal((12, V)) * 2.0).astype(np.float32)
+        u = rng.random(12).astype(np.float32)
+        r = oracle.sample_top_p(z, u, T, top_p)
+        p = _softmax64(z, T)
+        for i in range(12):
+            order = np.argsort(-p[i], kind="stable")
+            cum = np.cumsum(p[i][order])
+            k = int(np.searchsorted(cum, top_p, side="left")) + 1          # first prefix with mass >= top_p
+            keep = np.zeros(V, dtype=bool); keep[order[:k]] = True
+            q = np.where(keep, p[i], 0.0); q /= q.sum()
+            assert r["nucleus_size"][i] == k
+            np.testing.assert_allclose(r["q"][i], q, atol=1e-12)
+            if r["margin_sample"][i] > 1e-9:
+                assert r["token"][i] == int(np.searchsorted(np.cumsum(q), u[i] * 1.0, side="right"))
+            # the nucleus is minimal: without its least likely member the mass is below top_p
+            assert p[i][keep].sum() >= top_p - 1e-12 and p[i][keep].sum() - p[i][order[k - 1]] < top_p
+
+
+def test_top_p_limits():
+    """top_p = 1 keeps every token and is plain inverse-CDF sampling of softmax(z / T); a top_p below the
+    largest probability keeps only the argmax."""
+    rng = np.random.default_rng(6)
+    z = (rng.standard_normal((8, 50)) * 3.0).astype(np.float32)
+    u = rng.random(8).astype(np.float32)
+    full = oracle.sample_top_p(z, u, 0.8, 1.0)
+    p = _softmax64(z, 0.8)
+    assert np.all(full["nucleus_size"] == 50)
+    np.testing.assert_allclose(full["q"], p, atol=1e-12)
+    for i in range(8):
+        if full["margin_sample"][i] > 1e-9:
+            assert full["token"][i] == int(np.searchsorted(np.cumsum(p[i]), u[i] * p[i].sum(), side="right"))
+    greedy = oracle.sample_top_p(z, u, 0.8, 1e-6)
+    assert np.all(greedy["nucleus_size"] == 1) and np.array_equal(greedy["token"], p.argmax(-1))
+
+
+def test_top_p_marginal_is_the_renormalised_nucleus():
+    """Over a fine grid of uniforms the drawn tokens follow q (grid error at most 1/N per token) and
+    tokens outside the nucleus never appear."""
+    rng = np.random.default_rng(7)
+    z = (rng.standard_normal((1, 12)) * 1.5).astype(np.float32)
+    N = 4000
+    u = ((np.arange(N) + 0.5) / N).astype(np.float32)
+    r = oracle.sample_top_p(np.repeat(z, N, axis=0), u, 1.0, 0.8)
+    q = r["q"][0]
+    freq = np.bincount(r["token"], minlength=12) / N
+    assert np.all(np.abs(freq - q) <= 1.0 / N + 1e-12)
+    assert np.all(freq[q == 0] == 0)
