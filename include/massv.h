@@ -241,6 +241,27 @@ int massv_tvd(const massv_accept_desc *desc, const float *logits, const float *d
 int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t *accept_len, int32_t *seq_lens,
                     int32_t *dev_status, massv_stream_t stream);
 
+/*
+ * Nucleus (top-p) sampling of softmax(z / T), row by row (Sec. 3.2: the target's responses for the
+ * drafter's self-distillation are drawn as sample_top-p(p(. | I, X)); the same call is the drafter's
+ * sampling step when it samples with top-p, probs_out then being the draft distribution q that
+ * massv_accept takes).  Per row: order the tokens by probability, largest first (equal probabilities:
+ * lower index first); the nucleus is the shortest prefix of that order whose mass reaches top_p;
+ * q = p restricted to the nucleus and renormalised; tokens[r] is the inverse CDF of q in vocabulary
+ * order at u[r] (first index whose running mass exceeds u * total, never a zero-mass token).
+ *
+ *   rows, vocab   >= 1;  temperature > 0;  0 < top_p <= 1 (1 keeps every token)
+ *   logits        fp32 [rows, vocab] (for instance logits_out of massv_accept)
+ *   u             fp32 [rows], uniforms in [0, 1) supplied by the caller
+ *   tokens        int32 [rows]
+ *   probs_out     optional fp32 [rows, vocab]: q, zeros outside the nucleus
+ * Math: weights exp((z - max) / T) in fp32, all sums in fp64 in a fixed order.  No workspace.  A row
+ * without a finite logit stores MASSV_ERR_INVALID_ARG in dev_status and token 0.
+ */
+int massv_sample_top_p(int32_t rows, int32_t vocab, float temperature, float top_p, const float *logits,
+                       const float *u, int32_t *tokens, float *probs_out, int32_t *dev_status,
+                       massv_stream_t stream);
+
 /* Human-readable name of a massv_status value. */
 const char *massv_strerror(int status);
 

@@ -58,6 +58,8 @@ def _load():
     lib.massv_tvd_workspace_size.argtypes = [ctypes.POINTER(AcceptDesc)]
     lib.massv_tvd.restype = ctypes.c_int
     lib.massv_tvd.argtypes = [ctypes.POINTER(AcceptDesc), f32p, f32p, f32p, f32p, vp, ctypes.c_size_t, i32p, vp]
+    lib.massv_sample_top_p.restype = ctypes.c_int
+    lib.massv_sample_top_p.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_float, f32p, f32p, i32p, f32p, i32p, vp]
     lib.massv_kv_commit.restype = ctypes.c_int
     lib.massv_kv_commit.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, vp]
     lib.massv_strerror.restype = ctypes.c_char_p
@@ -195,6 +197,16 @@ def massv_tvd(desc, logits, draft_probs, tvd_out, accept_prob_out=None, workspac
                         _ptr(dev_status, torch.int32), _stream())
     if rc != 0:
         raise MassvError(rc, "massv_tvd")
+
+
+def massv_sample_top_p(logits, u, tokens, temperature, top_p, probs_out=None, dev_status=None) -> None:
+    """Nucleus sampling of softmax(logits / temperature), one draw per row (logits fp32 [rows, V])."""
+    f32, i32 = torch.float32, torch.int32
+    rows, vocab = logits.shape
+    rc = _lib.massv_sample_top_p(rows, vocab, float(temperature), float(top_p), _ptr(logits, f32), _ptr(u, f32),
+                                 _ptr(tokens, i32), _ptr(probs_out, f32), _ptr(dev_status, i32), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_sample_top_p")
 
 
 def massv_kv_commit(batch, gamma, accept_len, seq_lens, dev_status=None) -> None:

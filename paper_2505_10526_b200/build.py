@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG), "include")
 LIB = os.path.join(PKG, "libmassv.so")
-SOURCES = ["api.cu", "attn.cu", "attn_umma.cu", "lm_head.cu", "accept.cu", "accept_static.cu", "tensor_map.cu", "tvd.cu"]
+SOURCES = ["api.cu", "attn.cu", "attn_umma.cu", "lm_head.cu", "accept.cu", "accept_static.cu", "tensor_map.cu", "tvd.cu", "top_p.cu"]
 
 
 def _stale() -> bool:

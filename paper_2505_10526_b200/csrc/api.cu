@@ -241,6 +241,16 @@ int massv_tvd(const massv_accept_desc* desc, const float* logits, const float* d
     return launch_tvd(t, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
+int massv_sample_top_p(int32_t rows, int32_t vocab, float temperature, float top_p, const float* logits, const float* u,
+                       int32_t* tokens, float* probs_out, int32_t* dev_status, massv_stream_t stream) {
+    if (rows < 1 || vocab < 1 || !(temperature > 0.f) || !(top_p > 0.f) || !(top_p <= 1.f)) return MASSV_ERR_INVALID_ARG;
+    if (!logits || !u || !tokens) return MASSV_ERR_INVALID_ARG;
+    TopPParams t;
+    t.rows = rows; t.V = vocab; t.inv_T = 1.f / temperature; t.top_p = top_p;
+    t.logits = logits; t.u = u; t.tokens = tokens; t.probs_out = probs_out; t.dev_status = dev_status;
+    return launch_top_p(t, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
 int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
                     massv_stream_t stream) {
     if (batch < 1 || gamma < 0 || !seq_lens) return MASSV_ERR_INVALID_ARG;

@@ -93,6 +93,17 @@ struct TvdParams {
 };
 cudaError_t launch_tvd(const TvdParams& p, cudaStream_t stream);
 
+// ---------------------------------------------------------------- nucleus (top-p) sampling
+struct TopPParams {
+    int rows, V;
+    float inv_T, top_p;
+    const float *logits, *u;
+    int32_t* tokens;
+    float* probs_out;               // optional [rows, V]: the renormalised nucleus distribution
+    int32_t* dev_status;
+};
+cudaError_t launch_top_p(const TopPParams& p, cudaStream_t stream);
+
 cudaError_t launch_kv_commit(int B, int gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
                              cudaStream_t stream);
 

@@ -424,3 +424,80 @@ def test_batch_beyond_the_balanced_schedule_limit(kernel):
     cfg = VerifyConfig(name="big_batch", batch=1100, gamma=1, n_q_heads=4, n_kv_heads=2, head_dim=64, hidden=64, vocab=64,
                        temperature=0.0, ctx_lo=0, ctx_hi=90, image_tokens=0.25, draft_noise_std=0.5, seed=77)
     _attention_only_case(cfg, kernel)
+
+
+TOP_P_CASES = [
+    # rows, vocab, logit scale, temperature, top_p, quantise logits (forces many exactly equal probabilities)
+    (16, 1024, 2.0, 1.0, 0.9, False), (16, 1024, 2.0, 0.7, 0.5, False), (8, 1000, 4.0, 1.3, 0.25, False),
+    (8, 257, 1.0, 1.0, 1.0, False), (8, 4096, 3.0, 1.0, 1e-6, False), (12, 2048, 2.0, 1.0, 0.8, True),
+    (64, 152064, 1.5, 1.0, 0.95, False), (4, 152064, 6.0, 0.8, 0.5, False),
+]
+
+
+@pytest.mark.parametrize("rows,vocab,scale,T,top_p,quant", TOP_P_CASES)
+def test_top_p_sampling_matches_oracle(rows, vocab, scale, T, top_p, quant):
+    """massv_sample_top_p against the oracle's sort-based definition.  Nucleus membership (which entries
+    of probs_out are non-zero) and the drawn token are exact, except where the oracle's margins say the
+    decision is within rounding: the prefix mass that stops the nucleus within 1e-5 of top_p (fp32 weights
+    against fp64 ones), the uniform within 1e-3 of a CDF edge; q within 1e-4 absolute."""
+    import paper_2505_10526_b200 as mv
+    g = torch.Generator(device="cuda"); g.manual_seed(1000 + rows + vocab)
+    z = torch.randn((rows, vocab), generator=g, device="cuda", dtype=torch.float32) * scale
+    if quant:
+        z = torch.round(z * 2.0) / 2.0
+    u = torch.rand((rows,), generator=g, device="cuda", dtype=torch.float32)
+    tok = torch.full((rows,), -5, dtype=torch.int32, device="cuda")
+    q = torch.full((rows, vocab), -1.0, dtype=torch.float32, device="cuda")
+    status = torch.zeros((1,), dtype=torch.int32, device="cuda")
+    mv.massv_sample_top_p(z, u, tok, T, top_p, q, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = oracle.sample_top_p(z.cpu().numpy(), u.cpu().numpy(), T, top_p)
+    qg, tg = q.cpu().double().numpy(), tok.cpu().numpy()
+    exempt_set = exempt_draw = 0
+    for r in range(rows):
+        assert abs(qg[r].sum() - 1.0) < 1e-4 and qg[r].min() >= 0.0
+        if ref["margin_set"][r] < 1e-5 and not np.array_equal(qg[r] > 0, ref["q"][r] > 0):
+            exempt_set += 1
+            continue
+        # zero-probability members of the oracle's nucleus (top_p = 1 keeps everything) are not members here
+        assert np.array_equal(qg[r] > 0, ref["q"][r] > 0), (r, int((qg[r] > 0).sum()), int(ref["nucleus_size"][r]))
+        assert np.abs(qg[r] - ref["q"][r]).max() < TOL_PROB
+        if tg[r] != ref["token"][r]:
+            assert ref["margin_sample"][r] < 1e-3, (r, int(tg[r]), int(ref["token"][r]), float(ref["margin_sample"][r]))
+            exempt_draw += 1
+        assert qg[r][tg[r]] > 0
+    _report(dict(config=f"top_p rows={rows} V={vocab} T={T} p={top_p} quant={quant}", exempt_set=exempt_set, exempt_draw=exempt_draw))
+    assert exempt_set <= max(1, rows // 8)
+    # a second run is bit-identical
+    tok2 = torch.empty_like(tok); q2 = torch.empty_like(q)
+    mv.massv_sample_top_p(z, u, tok2, T, top_p, q2, status)
+    torch.cuda.synchronize()
+    assert torch.equal(tok, tok2) and torch.equal(q, q2)
+
+
+def test_top_p_output_feeds_the_acceptance_call():
+    """Drafter-side chain: logits from massv_accept (gamma = 0 rows), massv_sample_top_p for the drafts and
+    their distribution q, and q accepted as draft_probs by massv_accept: a drafter identical to the target
+    (same logits, T = 1, top_p = 1) has every draft accepted, since min(1, p/q) = 1."""
+    import paper_2505_10526_b200 as mv
+    cfg = get_config("tiny_peaked_t1")
+    w = generate(cfg, device="cuda", with_attention=False)
+    B, R, g, V = cfg.batch, cfg.rows, cfg.gamma, cfg.vocab
+    desc = mv.accept_desc(B, g, cfg.hidden, V, 1.0)
+    ws = mv.alloc_workspace(mv.massv_accept_workspace_size(desc), "cuda")
+    toks = torch.zeros((B, R), dtype=torch.int32, device="cuda"); lens = torch.zeros((B,), dtype=torch.int32, device="cuda")
+    logits = torch.zeros((B, R, V), dtype=torch.float32, device="cuda")
+    mv.massv_accept(desc, w["hidden"], w["lm_head"], w["draft_tokens"], w["draft_probs"], w["u_accept"], w["u_sample"],
+                    toks, lens, logits, None, ws, None)
+    z_draft = logits[:, :g].contiguous().view(B * g, V)
+    u = torch.rand((B * g,), device="cuda", dtype=torch.float32)
+    d_tok = torch.zeros((B * g,), dtype=torch.int32, device="cuda")
+    d_q = torch.zeros((B * g, V), dtype=torch.float32, device="cuda")
+    mv.massv_sample_top_p(z_draft, u, d_tok, 1.0, 1.0, d_q, None)
+    mv.massv_accept(desc, w["hidden"], w["lm_head"], d_tok.view(B, g).contiguous(), d_q.view(B, g, V), w["u_accept"], w["u_sample"],
+                    toks, lens, None, None, ws, None)
+    torch.cuda.synchronize()
+    # u * q < p fails only if rounding puts q above p by more than a factor 1/u: u is below 0.999 here
+    assert float(w["u_accept"].max()) < 0.9999
+    assert torch.all(lens == R) and torch.equal(toks[:, :g], d_tok.view(B, g))
