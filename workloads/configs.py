@@ -99,6 +99,7 @@ for _g in (5, 7):
 # acceptance call is the same, the attention part is small enough for multi-pass profiler captures.
 for _g in (3, 5, 7):
     _add(replace(CONFIGS[f"qwen7b_long_g{_g}_t0"], name=f"qwen7b_lmhead_g{_g}_t0", ctx_lo=64, ctx_hi=256, image_tokens=0.25))
+_add(replace(CONFIGS["qwen7b_long_g5_t1"], name="qwen7b_lmhead_g5_t1", ctx_lo=64, ctx_hi=256, image_tokens=0.25))
 
 
 def get_config(name: str) -> VerifyConfig:
