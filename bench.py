@@ -273,8 +273,8 @@ def main():
     assert int(step.dev_status.item()) == 0, "device-side error during the timed region"
 
     # ---- end to end: per-step inputs start in pinned host memory, results end there
-    host_inputs = {k: w[k].cpu().pin_memory() for k in STEP_KEYS if k in w and (cfg.temperature > 0 or k not in
-                   ("draft_probs", "u_accept", "u_sample"))}
+    host_inputs = step.host_inputs_like({k: w[k].cpu() for k in STEP_KEYS if k in w and (cfg.temperature > 0 or k not in
+                                         ("draft_probs", "u_accept", "u_sample"))})      # views of one pinned buffer
     resident = {k: w[k] for k in ("k_pages", "v_pages", "page_table", "seq_lens", "lm_head")}
     for _ in range(3):
         step.run_host(host_inputs, resident, commit=True)

@@ -31,8 +31,10 @@ class VerifyStep:
         self.attn_out = torch.empty((batch, self.R, n_q_heads, head_dim), dtype=torch.bfloat16, device=dev)
         self.attn_out_f32 = torch.empty_like(self.attn_out, dtype=torch.float32) if want_attn_f32 else None
         self.lse = torch.empty((batch, self.R, n_q_heads), dtype=torch.float32, device=dev) if want_attn_f32 else None
-        self.out_tokens = torch.empty((batch, self.R), dtype=torch.int32, device=dev)
-        self.accept_len = torch.empty((batch,), dtype=torch.int32, device=dev)
+        # tokens and accepted lengths share one buffer, so that a host reads both back with one copy
+        self._out_blob = torch.empty((batch * self.R + batch,), dtype=torch.int32, device=dev)
+        self.out_tokens = self._out_blob[:batch * self.R].view(batch, self.R)
+        self.accept_len = self._out_blob[batch * self.R:]
         self.logits = torch.empty((batch, self.R, vocab), dtype=torch.float32, device=dev) if want_logits else None
         self.probs = (torch.empty((batch, self.R, vocab), dtype=torch.float32, device=dev)
                       if want_probs and temperature > 0 else None)
@@ -70,25 +72,56 @@ class VerifyStep:
             self.commit(w["seq_lens"])
 
     # -- end-to-end step with host buffers ----------------------------------------------
+    def host_inputs_like(self, tensors):
+        """Pinned host buffers for the per-step inputs, shaped like ``tensors`` (a dict of name ->
+        tensor): views of ONE pinned allocation, mirrored by ONE device allocation, so that
+        ``run_host`` moves a step's inputs with a single copy however many tensors they are.  The
+        caller writes each step's inputs into the returned views in place."""
+        align = 256
+        layout, off = {}, 0
+        for k, v in tensors.items():
+            nbytes = v.numel() * v.element_size()
+            layout[k] = (off, nbytes, v.dtype, tuple(v.shape))
+            off = (off + nbytes + align - 1) // align * align
+        self._host_blob = torch.empty((max(off, align),), dtype=torch.uint8).pin_memory()
+        self._dev_blob = torch.empty((max(off, align),), dtype=torch.uint8, device=self.device)
+        view = lambda blob: {k: blob[o:o + n].view(dt).view(shape) for k, (o, n, dt, shape) in layout.items()}
+        self._host_views, self._staging = view(self._host_blob), view(self._dev_blob)
+        for k, v in tensors.items():
+            self._host_views[k].copy_(v)
+        self._host_out_blob = torch.empty(self._out_blob.shape, dtype=torch.int32).pin_memory()
+        n_tok = self.B * self.R
+        self._host_out = (self._host_out_blob[:n_tok].view(self.B, self.R), self._host_out_blob[n_tok:])
+        return self._host_views
+
     def run_host(self, host_inputs, resident, commit=False):
-        """One step whose per-step inputs start in pinned host memory and whose
-        result (tokens and accepted lengths) ends in pinned host memory.
-        Returns (out_tokens, accept_len) host tensors after synchronising."""
-        if self._staging is None:
-            self._staging = {k: torch.empty_like(v, device=self.device) for k, v in host_inputs.items()}
-            self._host_out = (torch.empty(self.out_tokens.shape, dtype=torch.int32).pin_memory(),
-                              torch.empty(self.accept_len.shape, dtype=torch.int32).pin_memory())
+        """One step whose per-step inputs start in pinned host memory and whose result (tokens and
+        accepted lengths) ends in pinned host memory.  ``host_inputs`` are the views returned by
+        ``host_inputs_like`` (one copy up, one copy down) or any dict of pinned tensors (one copy
+        per tensor).  Returns (out_tokens, accept_len) host tensors after synchronising."""
         w = dict(resident)
-        for k, v in host_inputs.items():
-            self._staging[k].copy_(v, non_blocking=True)
-            w[k] = self._staging[k]
+        if getattr(self, "_host_views", None) is not None and host_inputs is self._host_views:
+            self._dev_blob.copy_(self._host_blob, non_blocking=True)
+            w.update(self._staging)
+        else:
+            if self._staging is None or set(self._staging) != set(host_inputs):
+                self._staging = {k: torch.empty_like(v, device=self.device) for k, v in host_inputs.items()}
+            if self._host_out is None:
+                self._host_out_blob = torch.empty(self._out_blob.shape, dtype=torch.int32).pin_memory()
+                n_tok = self.B * self.R
+                self._host_out = (self._host_out_blob[:n_tok].view(self.B, self.R), self._host_out_blob[n_tok:])
+            for k, v in host_inputs.items():
+                self._staging[k].copy_(v, non_blocking=True)
+                w[k] = self._staging[k]
         self.run(w, commit=commit)
-        self._host_out[0].copy_(self.out_tokens, non_blocking=True)
-        self._host_out[1].copy_(self.accept_len, non_blocking=True)
+        self._host_out_blob.copy_(self._out_blob, non_blocking=True)
         torch.cuda.current_stream().synchronize()
         return self._host_out
 
     def host_bytes_per_step(self, host_inputs):
-        h2d = sum(v.numel() * v.element_size() for v in host_inputs.values())
+        if getattr(self, "_host_views", None) is not None and host_inputs is self._host_views:
+            h2d = self._host_blob.numel()           # the whole staging buffer goes up, padding included
+        else:
+            h2d = sum(v.numel() * v.element_size() for v in host_inputs.values())
         d2h = self.out_tokens.numel() * 4 + self.accept_len.numel() * 4
         return h2d, d2h

@@ -501,3 +501,28 @@ def test_top_p_output_feeds_the_acceptance_call():
     # u * q < p fails only if rounding puts q above p by more than a factor 1/u: u is below 0.999 here
     assert float(w["u_accept"].max()) < 0.9999
     assert torch.all(lens == R) and torch.equal(toks[:, :g], d_tok.view(B, g))
+
+
+@pytest.mark.parametrize("name", ["tiny_ragged_t1", "tiny_ragged_t0"])
+def test_host_staged_step_equals_the_device_resident_step(name):
+    """VerifyStep.run_host (inputs from pinned host memory, results to pinned host memory) returns what
+    the device-resident step returns, with the single staging buffer and with separate host tensors."""
+    from paper_2505_10526_b200 import VerifyStep
+    from paper_2505_10526_b200.step import STEP_INPUTS
+    cfg = get_config(name)
+    w = generate(cfg, device="cuda")
+    seq0 = w["seq_lens"].clone()
+    ref = VerifyStep.for_workload(cfg, w)
+    ref.run(w, commit=False)
+    torch.cuda.synchronize()
+    keys = [k for k in STEP_INPUTS if k in w and (cfg.temperature > 0 or k not in ("draft_probs", "u_accept", "u_sample"))]
+    resident = {k: w[k] for k in ("k_pages", "v_pages", "page_table", "seq_lens", "lm_head")}
+    one = VerifyStep.for_workload(cfg, w)
+    views = one.host_inputs_like({k: w[k].cpu() for k in keys})
+    toks, lens = one.run_host(views, resident, commit=False)
+    assert torch.equal(toks, ref.out_tokens.cpu()) and torch.equal(lens, ref.accept_len.cpu())
+    assert one.host_bytes_per_step(views)[0] >= sum(w[k].numel() * w[k].element_size() for k in keys)
+    many = VerifyStep.for_workload(cfg, w)
+    toks2, lens2 = many.run_host({k: w[k].cpu().pin_memory() for k in keys}, resident, commit=False)
+    assert torch.equal(toks2, ref.out_tokens.cpu()) and torch.equal(lens2, ref.accept_len.cpu())
+    assert torch.equal(w["seq_lens"], seq0)
