@@ -668,18 +668,28 @@ __global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(
     auto slot_of = [&](int i) -> size_t { const int c = c_first + i; return (size_t)c * 2 + (start <= c * per_cta ? 0 : 1); };
     // per row: the common maximum and 1 / sum; per (piece, row): the merge weight
     extern __shared__ float s_comb[];
-    float* s_w = s_comb;                           // [n][rows]
-    float* s_inv = s_comb + (size_t)n * rows;      // [rows]
+    float* s_w = s_comb;                           // [n][rows]: first the piece maxima, then the merge weights
+    float* s_l = s_comb + (size_t)n * rows;        // [n][rows]: the pieces' sums
+    float* s_inv = s_comb + 2 * (size_t)n * rows;  // [rows]
+    // every (piece, row) pair's (max, sum) with one load per thread: a pair cut into dozens of pieces
+    // must not walk them one latency after the other
+    for (int idx = threadIdx.x; idx < n * rows; idx += blockDim.x) {
+        const int i = idx / rows, rr = idx % rows;
+        const float2 ml = *reinterpret_cast<const float2*>(p.flat_part_ml + (slot_of(i) * rows_pad + row0 + rr) * 2);
+        s_w[idx] = ml.x;
+        s_l[idx] = ml.y;
+    }
+    __syncthreads();
     for (int rr = threadIdx.x; rr < rows; rr += blockDim.x) {
         const int r = row0 + rr;
         float M = -INFINITY;
-        for (int i = 0; i < n; ++i) M = fmaxf(M, p.flat_part_ml[(slot_of(i) * rows_pad + r) * 2]);
+        for (int i = 0; i < n; ++i) M = fmaxf(M, s_w[(size_t)i * rows + rr]);
         float Lsum = 0.f;
         for (int i = 0; i < n; ++i) {
-            const float2 ml = *reinterpret_cast<const float2*>(p.flat_part_ml + (slot_of(i) * rows_pad + r) * 2);
-            const float w = ml.x == -INFINITY ? 0.f : exp2f(ml.x - M);
+            const float mi = s_w[(size_t)i * rows + rr];
+            const float w = mi == -INFINITY ? 0.f : exp2f(mi - M);
             s_w[(size_t)i * rows + rr] = w;
-            Lsum += ml.y * w;
+            Lsum += s_l[(size_t)i * rows + rr] * w;
         }
         s_inv[rr] = 1.f / Lsum;
         if (p.lse) p.lse[((size_t)b * p.R + r / G) * p.Hq + g * G + r % G] = (M + log2f(Lsum)) * 0.6931471805599453f;
@@ -743,14 +753,14 @@ cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtens
         if (e != cudaSuccess) return e;
         if (split_done && cudaEventRecord(split_done, stream) != cudaSuccess) return cudaGetLastError();
         const int rows = (p.Hq / p.Hkv) * p.R;
-        // weights for at most `ctas` pieces of a pair (a pair can span every CTA), plus one value per row
+        // (max, sum) and weight for at most `ctas` pieces of a pair (a pair can span every CTA), plus one value per row
         // enough CTAs to fill the machine: a pair's rows are dealt to several CTAs when there are few pairs
         const int pairs = p.B * p.Hkv;
         int row_groups = (2 * flat_sm_count() + pairs - 1) / pairs;
         if (row_groups > rows) row_groups = rows;
         const int rows_per_cta = (rows + row_groups - 1) / row_groups;
         row_groups = (rows + rows_per_cta - 1) / rows_per_cta;
-        const size_t comb_smem = ((size_t)ctas + 1) * rows_per_cta * sizeof(float);
+        const size_t comb_smem = (2 * (size_t)ctas + 1) * rows_per_cta * sizeof(float);
         e = cudaFuncSetAttribute(attn_flat_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)comb_smem);
         if (e != cudaSuccess) return e;
         const int threads = rows_per_cta * (p.d / 4) <= 64 ? 64 : (rows_per_cta * (p.d / 4) <= 128 ? 128 : kFlatCombineThreads);
