@@ -250,7 +250,7 @@ int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t *accept_len, int
  * q = p restricted to the nucleus and renormalised; tokens[r] is the inverse CDF of q in vocabulary
  * order at u[r] (first index whose running mass exceeds u * total, never a zero-mass token).
  *
- *   rows, vocab   >= 1;  temperature > 0;  0 < top_p <= 1 (1 keeps every token)
+ *   rows >= 1;  1 <= vocab <= 2^21;  temperature > 0;  0 < top_p <= 1 (1 keeps every token)
  *   logits        fp32 [rows, vocab] (for instance logits_out of massv_accept)
  *   u             fp32 [rows], uniforms in [0, 1) supplied by the caller
  *   tokens        int32 [rows]

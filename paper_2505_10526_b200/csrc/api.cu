@@ -245,6 +245,7 @@ int massv_sample_top_p(int32_t rows, int32_t vocab, float temperature, float top
                        int32_t* tokens, float* probs_out, int32_t* dev_status, massv_stream_t stream) {
     if (rows < 1 || vocab < 1 || !(temperature > 0.f) || !(top_p > 0.f) || !(top_p <= 1.f)) return MASSV_ERR_INVALID_ARG;
     if (!logits || !u || !tokens) return MASSV_ERR_INVALID_ARG;
+    if (vocab > (1 << 21)) return MASSV_ERR_UNSUPPORTED;
     TopPParams t;
     t.rows = rows; t.V = vocab; t.inv_T = 1.f / temperature; t.top_p = top_p;
     t.logits = logits; t.u = u; t.tokens = tokens; t.probs_out = probs_out; t.dev_status = dev_status;

@@ -56,11 +56,17 @@ __device__ __forceinline__ unsigned long long block_suffix_exclusive_u64(unsigne
 
 constexpr int kTopPBins = 512;      // 9 bits of the pattern per level (9 + 9 + 9 + 4)
 constexpr int kTopPCopies = 8;
+constexpr int kTopPMaxBlocks = kTopPBins * kTopPCopies / kTopPWarps;     // 512-entry blocks per warp: 128, i.e. V <= 2^21
 
 __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
     const int row = blockIdx.x, t = threadIdx.x;
     const float* z = p.logits + (size_t)row * p.V;
-    __shared__ uint32_t hist_lo[kTopPBins * kTopPCopies], hist_hi[kTopPBins * kTopPCopies];
+    // 32 KB used twice: the histograms' low and high words during the threshold search, then the masses
+    // of the 512-entry blocks of every warp's range
+    __shared__ __align__(16) unsigned long long pool[kTopPBins * kTopPCopies];
+    uint32_t* hist_lo = reinterpret_cast<uint32_t*>(pool);
+    uint32_t* hist_hi = hist_lo + kTopPBins * kTopPCopies;
+    double* block_mass = reinterpret_cast<double*>(pool);          // [kTopPWarps][kTopPMaxBlocks]
     __shared__ unsigned long long sm_u64[kTopPWarps];
     __shared__ int s_bin;
     __shared__ unsigned long long s_above;
@@ -116,14 +122,29 @@ __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
         const int sh = e - 127 - 23 + fx_bits;             // w = mant * 2^(e - 127 - 23)
         return sh >= 0 ? mant << sh : (sh > -24 ? mant >> (-sh) : 0ull);
     };
-    unsigned long long local = 0ull;
+    // the same number as two 32-bit words, from two float -> integer conversions (fx_bits == 44):
+    // hi = floor(w * 2^12), lo = floor((w - hi * 2^-12) * 2^44); both products and the difference are exact
+    auto fixed_words = [&](float w, uint32_t& hi, uint32_t& lo) {
+        if (fx_bits == 44) {
+            hi = __float2uint_rz(w * 4096.f);
+            lo = __float2uint_rz(fmaf(-(float)hi, 1.f / 4096.f, w) * 17592186044416.f);
+        } else {
+            const unsigned long long f = fixed(w);
+            hi = (uint32_t)(f >> 32); lo = (uint32_t)f;
+        }
+    };
+    unsigned long long local_hi = 0ull, local_lo = 0ull;
     for (int v = t; v < p.V; v += kUnroll * kTopPThreads) {
         float zz[kUnroll];
         load4(v, kTopPThreads, zz);
 #pragma unroll
-        for (int j = 0; j < kUnroll; ++j) local += fixed(weight_of(zz[j]));
+        for (int j = 0; j < kUnroll; ++j) {
+            uint32_t hi, lo;
+            fixed_words(weight_of(zz[j]), hi, lo);
+            local_hi += hi; local_lo += lo;
+        }
     }
-    const unsigned long long S_fx = block_sum_u64(local, sm_u64);
+    const unsigned long long S_fx = (block_sum_u64(local_hi, sm_u64) << 32) + block_sum_u64(local_lo, sm_u64);
     unsigned long long target_fx = (unsigned long long)ceil((double)p.top_p * (double)S_fx);
     if (target_fx > S_fx) target_fx = S_fx;
     if (target_fx == 0ull) target_fx = 1ull;
@@ -150,14 +171,11 @@ __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
                 const float w = weight_of(zz[j]);
                 const uint32_t b = __float_as_uint(w);
                 if ((b & hi_mask) == prefix) {
-                    const unsigned long long f = fixed(w);
-                    if (f) {
-                        const int bin = my_copy + (int)((b >> shift) & (uint32_t)(nbins - 1));
-                        const uint32_t lo = (uint32_t)f;
-                        uint32_t hi = (uint32_t)(f >> 32);
-                        if (lo) hi += (atomicAdd(&hist_lo[bin], lo) > ~lo) ? 1u : 0u;      // the low word wrapped
-                        if (hi) atomicAdd(&hist_hi[bin], hi);
-                    }
+                    uint32_t hi, lo;
+                    fixed_words(w, hi, lo);
+                    const int bin = my_copy + (int)((b >> shift) & (uint32_t)(nbins - 1));
+                    if (lo) hi += (atomicAdd(&hist_lo[bin], lo) > ~lo) ? 1u : 0u;      // the low word wrapped
+                    if (hi) atomicAdd(&hist_hi[bin], hi);
                 }
             }
         }
@@ -211,13 +229,17 @@ __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
     __syncthreads();
     long long tie_base = 0;
     for (int w = 0; w < warp; ++w) tie_base += warp_ties[w];
-    // mass per warp (members only), summed round by round
+    // mass per warp (members only): per block of 16 rounds (512 entries) every lane adds up its own
+    // entries, then one warp-wide sum; the block masses are kept for the draw
+    __syncthreads();                             // the histograms are not read any more: the pool changes hands
     {
         long long rank0 = tie_base;              // ties before the current round
         double acc = 0.0;
-        for (int v = w0 + lane; v - lane < w1; v += kUnroll * 32) {
+        int blk = 0;
+        for (int v = w0 + lane; v - lane < w1; v += kUnroll * 32, ++blk) {
             float zz[kUnroll];
             load4(v, 32, zz);
+            double x = 0.0;
 #pragma unroll
             for (int j = 0; j < kUnroll; ++j) {
                 const float w = (v + j * 32 < w1) ? weight_of(zz[j]) : 0.f;
@@ -226,11 +248,12 @@ __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
                 const unsigned ties = __ballot_sync(0xffffffffu, tie);
                 const bool in = (v + j * 32 < w1) && (b > tau || (tie && rank0 + __popc(ties & lt_mask) < n_ties));
                 rank0 += __popc(ties);
-                double x = in ? (double)w : 0.0;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-                acc += x;
+                if (in) x += (double)w;
             }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if (lane == 0) block_mass[warp * kTopPMaxBlocks + blk] = x;
+            acc += x;
         }
         if (lane == 0) warp_mass[warp] = acc;
     }
@@ -248,11 +271,17 @@ __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
     const float inv_Z = (float)(1.0 / Z);
     {
         long long rank0 = tie_base;
-        double run = base;                       // mass before the current round
+        double run = base;                       // mass before the current block / round
         int first = 0x7fffffff, last = -1;
-        for (int v = w0 + lane; v - lane < w1; v += kUnroll * 32) {
+        int blk = 0;
+        for (int v = w0 + lane; v - lane < w1; v += kUnroll * 32, ++blk) {
             float zz[kUnroll];
             load4(v, 32, zz);
+            // only the block that holds the target is walked round by round with running sums
+            const double blk_mass = block_mass[warp * kTopPMaxBlocks + blk];
+            const bool scan = holds && first == 0x7fffffff && blk_mass > 0.0 && run <= target && target < run + blk_mass;
+            double run_in = run;
+            int blk_last = -1;
 #pragma unroll
             for (int j = 0; j < kUnroll; ++j) {
                 const int vv = v + j * 32;
@@ -263,7 +292,8 @@ __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
                 const bool in = vv < w1 && w > 0.f && (b > tau || (tie && rank0 + __popc(ties & lt_mask) < n_ties));
                 rank0 += __popc(ties);
                 if (p.probs_out && vv < w1) p.probs_out[(size_t)row * p.V + vv] = in ? w * inv_Z : 0.f;
-                if (holds || last_with_mass) {
+                if (in) { last = vv; blk_last = vv; }
+                if (scan) {
                     // inclusive sum over the lanes of this round, in lane order
                     double incl = in ? (double)w : 0.0;
 #pragma unroll
@@ -271,19 +301,21 @@ __global__ void __launch_bounds__(kTopPThreads) top_p_kernel(TopPParams p) {
                         const double y = __shfl_up_sync(0xffffffffu, incl, o);
                         if (lane >= o) incl += y;
                     }
-                    if (in) {
-                        last = vv;
-                        if (first == 0x7fffffff && run + incl > target) first = vv;
-                    }
-                    run += __shfl_sync(0xffffffffu, incl, 31);
+                    if (in && first == 0x7fffffff && run_in + incl > target) first = vv;
+                    run_in += __shfl_sync(0xffffffffu, incl, 31);
                 }
             }
+            if (scan) {
+                // (the round sums and the block's mass add the same numbers in another order: if the last bit
+                // puts the target past the running sum, the block's last member is the answer)
+                first = __reduce_min_sync(0xffffffffu, first);
+                if (first == 0x7fffffff) first = __reduce_max_sync(0xffffffffu, blk_last);
+            }
+            run += blk_mass;
         }
         first = __reduce_min_sync(0xffffffffu, first);
         last = __reduce_max_sync(0xffffffffu, last);
-        // (the round sums here and the warp's total above add the same numbers in another order: if the
-        // last bit puts the target past this warp's own running sum, its last member is the answer)
-        if (holds && first == 0x7fffffff && last >= 0) first = last;
+        if (holds && first == 0x7fffffff && last >= 0) first = last;      // no block claimed the target (rounding): the warp's last member
         if (holds && first != 0x7fffffff) atomicMin(&s_first, first);
         if (last_with_mass && last >= 0) atomicMax(&s_last, last);
     }
