@@ -302,6 +302,16 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             const int n_pages = (sg.c_end - sg.c_begin + kPageSize - 1) / kPageSize;
             int pid_prev = 0, pid_cur = lane < n_pages ? pt[lane] : 0, pid_next = 32 + lane < n_pages ? pt[32 + lane] : 0;
             int grp_cur = 0;
+            if (sg.c_end > L) {
+                // the segment ends with the block's own positions: bring the block's K/V rows into L2 now, so
+                // that the patches at its end do not each wait for a cold load
+                constexpr int LPR = D / 64;               // 128-byte lines per row
+                for (int i = lane; i < 2 * p.R * LPR; i += 32) {
+                    const int pv = i / (p.R * LPR), j = (i / LPR) % p.R, c = i % LPR;
+                    const __nv_bfloat16* src = (pv ? p.v_new : p.k_new) + (((size_t)b * p.R + j) * p.Hkv + g) * D + c * 64;
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
+                }
+            }
             for (int i = 0; i < 2 * n_tiles; ++i, ++it) {
                 // item i of the consumption order: which tile, and whether its K or its V
                 int t, is_v;
