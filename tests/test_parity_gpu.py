@@ -383,13 +383,13 @@ def test_timing_hook_brackets_the_dominant_kernels():
     assert ev[1].elapsed_time(ev[2]) == lm          # not re-recorded once the hook is off
 
 
-def _attention_only_case(cfg, kernel, kv_chunk=0):
+def _attention_only_case(cfg, kernel, kv_chunk=0, window=0):
     """massv_verify_attn alone (no LM head) against the oracle's attention, for shapes whose
     acceptance part would be out of range or beside the point."""
     from paper_2505_10526_b200 import VerifyStep
     w = generate(cfg, device="cuda")
     before = {k: w[k].clone() for k in ("k_pages", "v_pages", "seq_lens")}
-    step = VerifyStep.for_workload(cfg, w, want_attn_f32=True, attn_kernel=kernel, kv_chunk=kv_chunk)
+    step = VerifyStep.for_workload(cfg, w, want_attn_f32=True, attn_kernel=kernel, kv_chunk=kv_chunk, window=window)
     step.attn(w)
     torch.cuda.synchronize()
     assert int(step.dev_status.item()) == 0
@@ -398,7 +398,7 @@ def _attention_only_case(cfg, kernel, kv_chunk=0):
     pt = w["page_table"].cpu().numpy().astype(np.int32)
     seq = before["seq_lens"].cpu().numpy().astype(np.int32)
     oracle.kv_append(oracle.bf16_bits(w["k_new"]), oracle.bf16_bits(w["v_new"]), kp, vp, pt, seq)
-    out, lse = oracle.verify_attn(oracle.bf16_bits(w["q"]), kp, vp, pt, seq)
+    out, lse = oracle.verify_attn(oracle.bf16_bits(w["q"]), kp, vp, pt, seq, window=window)
     ref = dict(attn_out=out, lse=lse, k_pages=kp, v_pages=vp)
     err = float(np.abs(step.attn_out_f32.cpu().double().numpy() - ref["attn_out"]).max())
     err16 = float(np.abs(step.attn_out.cpu().double().numpy() - ref["attn_out"]).max())
@@ -527,3 +527,46 @@ def test_host_staged_step_equals_the_device_resident_step(name):
     toks2, lens2 = many.run_host({k: w[k].cpu().pin_memory() for k in keys}, resident, commit=False)
     assert torch.equal(toks2, ref.out_tokens.cpu()) and torch.equal(lens2, ref.accept_len.cpu())
     assert torch.equal(w["seq_lens"], seq0)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_attention_on_random_small_shapes(seed):
+    """Seeded random geometry: heads, group size, head_dim, gamma, context ranges that start at zero,
+    sliding windows and forced chunk sizes, each through both split kernels."""
+    import random
+    from workloads import VerifyConfig
+    rnd = random.Random(9000 + seed)
+    d = rnd.choice([64, 128, 128, 256])
+    gamma = rnd.randint(0, 7)
+    n_kv = rnd.choice([1, 2, 4])
+    group = rnd.randint(1, max(1, min(8, 64 // (gamma + 1))))
+    ctx_hi = rnd.choice([40, 150, 333, 700])
+    cfg = VerifyConfig(name=f"fuzz{seed}", batch=rnd.randint(1, 6), gamma=gamma, n_q_heads=n_kv * group, n_kv_heads=n_kv,
+                       head_dim=d, hidden=64, vocab=64, temperature=0.0, ctx_lo=rnd.choice([0, 0, ctx_hi // 2]), ctx_hi=ctx_hi,
+                       image_tokens=0.25, draft_noise_std=0.5, seed=9000 + seed)
+    window = rnd.choice([0, 0, 1, 17, 64, 200])
+    kv_chunk = rnd.choice([0, 0, 64, 128])
+    for kernel in (1, 2):
+        _attention_only_case(cfg, kernel, kv_chunk=kv_chunk, window=window)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_whole_step_on_random_small_shapes(seed):
+    """Seeded random geometry for the whole step: vocabulary sizes off the 128-row tile, hidden sizes of
+    one to nine K blocks, row counts from 1 to a few hundred (single CTAs and CTA pairs in the LM head),
+    greedy and sampled verification."""
+    import random
+    from workloads import VerifyConfig
+    rnd = random.Random(7000 + seed)
+    gamma = rnd.randint(0, 7)
+    batch = rnd.choice([1, 2, 3, 5, 9, 17, 40])
+    while batch * (gamma + 1) > 320:
+        batch //= 2
+    n_kv = rnd.choice([1, 2])
+    group = rnd.randint(1, max(1, min(4, 64 // (gamma + 1))))
+    cfg = VerifyConfig(name=f"stepfuzz{seed}", batch=batch, gamma=gamma, n_q_heads=n_kv * group, n_kv_heads=n_kv,
+                       head_dim=rnd.choice([64, 128]), hidden=64 * rnd.randint(1, 9), vocab=8 * rnd.randint(40, 1500),
+                       temperature=rnd.choice([0.0, 0.0, 0.6, 1.0, 1.4]), ctx_lo=0, ctx_hi=rnd.choice([30, 120, 300]),
+                       image_tokens=0.25, draft_noise_std=rnd.choice([0.3, 1.0]), seed=7000 + seed,
+                       hidden_std=rnd.choice([1.0, 6.0]))
+    run_case(None, cfg=cfg, check_determinism=(seed % 4 == 0))
