@@ -95,9 +95,9 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
         } else if (greedy) {
             ok = (x == row_stat[lane].idx);
         } else {
-            const float zx = p.logits[(size_t)(b * R + lane) * p.V + x];
+            const float zx = p.z_at_draft ? p.z_at_draft[(size_t)b * p.gamma + lane] : p.logits[(size_t)(b * R + lane) * p.V + x];
             const float px = expf((zx - row_stat[lane].m) * inv_T) / row_stat[lane].s;
-            const float qx = p.draft_probs[((size_t)b * p.gamma + lane) * p.V + x];
+            const float qx = p.q_at_draft ? p.q_at_draft[(size_t)b * p.gamma + lane] : p.draft_probs[((size_t)b * p.gamma + lane) * p.V + x];
             const float lhs = p.u_accept[(size_t)b * p.gamma + lane] * qx;
             ok = lhs < px;
         }
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
         st.row_max = row_stat[n].m;
         st.inv_sum = 1.f / row_stat[n].s;
         p.seq_state[b] = st;
-        p.counters[b] = 0u;
+        if (p.counters) p.counters[b] = 0u;
     }
 }
 
@@ -286,6 +286,163 @@ __global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptP
     if (t == 0) *tok_out = (!take_last && s_first != 0x7fffffff) ? s_first : s_last;
 }
 
+// ---------------------------------------------------------------- vocabulary shards
+// The same arithmetic with the vocabulary cut into contiguous shards, one per rank: a shard sees Vs
+// columns of the logits and of q.  Chunks are counted inside the shard; ranks in order are vocabulary order.
+
+// Masses of the 16 entries this thread owns in chunk c of the sampled row of a shard.
+__device__ __forceinline__ void shard_chunk_masses(const ShardParams& p, int b, const SeqState& st, int use_q, int c,
+                                                   float inv_T, float (&r)[kPerThread]) {
+    const int R = p.gamma + 1;
+    const int v0 = c * kResidualChunk + threadIdx.x * kPerThread;
+    const float* z = p.logits + (size_t)(b * R + st.n) * p.Vs;
+    const float* q = use_q ? p.draft_probs + ((size_t)b * p.gamma + st.n) * p.Vs : nullptr;
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) {
+        const int v = v0 + e;
+        float m = 0.f;
+        if (v < p.Vs) {
+            const float pv = expf((z[v] - st.row_max) * inv_T) * st.inv_sum;
+            m = q ? fmaxf(pv - q[v], 0.f) : pv;
+        }
+        r[e] = m;
+    }
+}
+
+// Logit and drafter probability at each drafted token this shard owns (-inf elsewhere: a maximum
+// over the ranks then yields the owner's values).
+__global__ void shard_gather_draft_kernel(ShardParams p) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait();
+    if (i >= p.B * p.gamma) return;
+    const int b = i / p.gamma, j = i % p.gamma, R = p.gamma + 1;
+    const int x = p.draft_tokens[i] - p.vocab_offset;
+    const bool mine = x >= 0 && x < p.Vs;
+    p.z_at_draft[i] = mine ? p.logits[(size_t)(b * R + j) * p.Vs + x] : -INFINITY;
+    if (p.q_at_draft) p.q_at_draft[i] = mine ? p.draft_probs[((size_t)b * p.gamma + j) * p.Vs + x] : -INFINITY;
+}
+
+// grid (n_chunks, B): the shard's chunk masses of the residual max(p - q, 0) and of p on the sampled row.
+__global__ void __launch_bounds__(kSampleThreads) shard_masses_kernel(ShardParams p) {
+    const int c = blockIdx.x, b = blockIdx.y, t = threadIdx.x;
+    const float inv_T = 1.f / p.T;
+    pdl_wait();
+    pdl_trigger();
+    const SeqState st = p.seq_state[b];
+    __shared__ double warp_sums[kSampleThreads / 32];
+    float r[kPerThread];
+    for (int pass = 0; pass < 2; ++pass) {
+        // pass 0: the distribution the extra token is drawn from; pass 1: p itself (the fall-back when
+        // the residual has no mass anywhere)
+        const int use_q = pass == 0 ? st.use_q : 0;
+        shard_chunk_masses(p, b, st, use_q, c, inv_T, r);
+        double local = 0.0;
+#pragma unroll
+        for (int e = 0; e < kPerThread; ++e) local += (double)r[e];
+        double total;
+        block_exclusive_scan(local, warp_sums, &total);
+        if (t == 0) (pass == 0 ? p.sums_res : p.sums_p)[(size_t)b * p.n_chunks + c] = total;
+        if (pass == 0 && !st.use_q) {          // the two passes coincide
+            if (t == 0) p.sums_p[(size_t)b * p.n_chunks + c] = total;
+            break;
+        }
+    }
+}
+
+// One CTA per sequence.  Every rank walks the same chunk masses of all shards; the rank whose shard holds
+// the winning chunk finds the token inside it, the others store -1.
+__global__ void __launch_bounds__(kSampleThreads) shard_pick_kernel(ShardParams p) {
+    const int b = blockIdx.x, t = threadIdx.x;
+    const int R = p.gamma + 1, n_all = p.world * p.n_chunks;
+    const float inv_T = 1.f / p.T;
+    pdl_wait();
+    pdl_trigger();
+    const SeqState st = p.seq_state[b];
+    __shared__ double warp_sums[kSampleThreads / 32];
+    __shared__ double s_sums[kWalkChunks];
+    __shared__ int s_pick[3];
+    __shared__ double s_base[2];
+    __shared__ int s_first, s_last;
+    if (n_all > kWalkChunks) {
+        if (t == 0) { p.token_out[b] = -1; set_status(p.dev_status, MASSV_ERR_UNSUPPORTED); }
+        return;
+    }
+    int use_q = st.use_q;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        // gathered layout [world, B, n_chunks]: rank r's chunks of sequence b are contiguous
+        const double* sums = use_q ? p.all_res : p.all_p;
+        for (int i = t; i < n_all; i += kSampleThreads)
+            s_sums[i] = sums[((size_t)(i / p.n_chunks) * p.B + b) * p.n_chunks + i % p.n_chunks];
+        __syncthreads();
+        if (t == 0) {
+            double tot = 0.0;
+            for (int i = 0; i < n_all; ++i) tot += s_sums[i];
+            const double target = (double)p.u_sample[(size_t)b * R + st.n] * tot;
+            int pick = -1, last_pos = -1;
+            double cum = 0.0, base = 0.0;
+            for (int i = 0; i < n_all; ++i) {
+                const double s = s_sums[i];
+                if (s > 0.0) last_pos = i;
+                if (pick < 0 && s > 0.0 && cum + s > target) { pick = i; base = cum; }
+                cum += s;
+            }
+            s_pick[0] = tot > 0.0 ? (pick >= 0 ? pick : last_pos) : -1;
+            s_pick[1] = (pick < 0);
+            s_base[0] = base;
+            s_base[1] = target;
+        }
+        __syncthreads();
+        if (s_pick[0] >= 0 || !use_q) break;
+        use_q = 0;                             // the residual has no mass (p == q on this row): draw from p
+        __syncthreads();
+    }
+    const int pick = s_pick[0];
+    if (pick < 0) {
+        if (t == 0) { p.token_out[b] = p.rank == 0 ? 0 : -1; set_status(p.dev_status, MASSV_ERR_INVALID_ARG); }
+        return;
+    }
+    if (pick / p.n_chunks != p.rank) {         // another shard holds the chunk
+        if (t == 0) p.token_out[b] = -1;
+        return;
+    }
+    const int c = pick % p.n_chunks;
+    const bool take_last = s_pick[1] != 0;
+    const double base = s_base[0], target = s_base[1];
+    float r[kPerThread];
+    shard_chunk_masses(p, b, st, use_q, c, inv_T, r);
+    double loc = 0.0;
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) loc += (double)r[e];
+    double tt;
+    double run = base + block_exclusive_scan(loc, warp_sums, &tt);
+    int first = 0x7fffffff, last = -1;
+#pragma unroll
+    for (int e = 0; e < kPerThread; ++e) {
+        run += (double)r[e];
+        if (r[e] > 0.f) {
+            const int v = c * kResidualChunk + t * kPerThread + e;
+            last = v;
+            if (first == 0x7fffffff && run > target) first = v;
+        }
+    }
+    if (t == 0) { s_first = 0x7fffffff; s_last = -1; }
+    __syncthreads();
+    atomicMin(&s_first, first);
+    atomicMax(&s_last, last);
+    __syncthreads();
+    if (t == 0) p.token_out[b] = p.vocab_offset + ((!take_last && s_first != 0x7fffffff) ? s_first : s_last);
+}
+
+// The extra token, once the ranks have agreed on it, goes to its place after the accepted drafts.
+__global__ void shard_set_token_kernel(ShardParams p) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait();
+    if (b >= p.B) return;
+    const int tok = p.tokens_in[b];
+    if (tok < 0) { set_status(p.dev_status, MASSV_ERR_INVALID_ARG); return; }
+    p.out_tokens[(size_t)b * (p.gamma + 1) + p.seq_state[b].n] = tok;
+}
+
 // Dense probabilities for callers that ask for them (diagnostics / tests).
 __global__ void probs_kernel(AcceptParams p) {
     const int R = p.gamma + 1, M = p.B * R;
@@ -336,6 +493,35 @@ cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream) {
             count_launches(1);
         }
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accept_scan_only(const AcceptParams& p, cudaStream_t stream) {
+    if (launch_pdl(accept_scan_kernel, dim3(p.B), dim3(kScanThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_gather_draft(const ShardParams& p, cudaStream_t stream) {
+    const int n = p.B * p.gamma;
+    if (n == 0) return cudaSuccess;
+    if (launch_pdl(shard_gather_draft_kernel, dim3((n + 127) / 128), dim3(128), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
+    return cudaGetLastError();
+}
+cudaError_t launch_shard_masses(const ShardParams& p, cudaStream_t stream) {
+    if (launch_pdl(shard_masses_kernel, dim3(p.n_chunks, p.B), dim3(kSampleThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
+    return cudaGetLastError();
+}
+cudaError_t launch_shard_pick(const ShardParams& p, cudaStream_t stream) {
+    if (launch_pdl(shard_pick_kernel, dim3(p.B), dim3(kSampleThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
+    return cudaGetLastError();
+}
+cudaError_t launch_shard_set_token(const ShardParams& p, cudaStream_t stream) {
+    if (launch_pdl(shard_set_token_kernel, dim3((p.B + 127) / 128), dim3(128), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
     return cudaGetLastError();
 }
 

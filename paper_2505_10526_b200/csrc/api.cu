@@ -212,6 +212,143 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
     return launch_accept(a, s) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
+// ---------------------------------------------------------------- vocabulary shards
+size_t massv_shard_max_partials(const massv_accept_desc* desc) {
+    if (check_accept_desc(desc) != MASSV_OK) return 0;
+    return (size_t)lm_head_num_partials(desc->batch * (desc->gamma + 1), desc->vocab);
+}
+
+size_t massv_shard_chunks(const massv_accept_desc* desc) {
+    if (check_accept_desc(desc) != MASSV_OK) return 0;
+    return (size_t)((desc->vocab + kResidualChunk - 1) / kResidualChunk);
+}
+
+size_t massv_shard_state_bytes(const massv_accept_desc* desc) {
+    if (check_accept_desc(desc) != MASSV_OK) return 0;
+    return (size_t)desc->batch * sizeof(SeqState);
+}
+
+static int check_shard(const massv_accept_desc* desc, int32_t world, int32_t rank) {
+    const int rc = check_accept_desc(desc);
+    if (rc != MASSV_OK) return rc;
+    if (world < 1 || rank < 0 || rank >= world) return MASSV_ERR_INVALID_ARG;
+    if ((long)world * desc->vocab > 0x7fffffffL) return MASSV_ERR_UNSUPPORTED;
+    return MASSV_OK;
+}
+
+int massv_shard_lm_head(const massv_accept_desc* desc, int32_t world, int32_t rank, const void* hidden,
+                        const void* lm_head_shard, float* logits_shard, float* part_max, float* part_sum,
+                        int32_t* part_idx, int32_t* n_partials, int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_shard(desc, world, rank);
+    if (rc != MASSV_OK) return rc;
+    const bool sampling = desc->temperature > 0.f;
+    if (!hidden || !lm_head_shard || !part_max || !part_sum || !part_idx || !n_partials) return MASSV_ERR_INVALID_ARG;
+    if (sampling && !logits_shard) return MASSV_ERR_INVALID_ARG;
+    if (!aligned16(hidden) || !aligned16(lm_head_shard) || (logits_shard && !aligned16(logits_shard)))
+        return MASSV_ERR_INVALID_ARG;
+    LmHeadParams g;
+    g.M = desc->batch * (desc->gamma + 1); g.K = desc->hidden; g.V = desc->vocab;
+    g.greedy = sampling ? 0 : 1;
+    g.inv_T_log2e = sampling ? 1.4426950408889634f / desc->temperature : 0.f;
+    g.hidden = static_cast<const __nv_bfloat16*>(hidden);
+    g.lm_head = static_cast<const __nv_bfloat16*>(lm_head_shard);
+    g.logits = logits_shard;
+    g.n_part = lm_head_num_partials(g.M, g.V);
+    g.part_max = part_max; g.part_sum = part_sum; g.part_idx = part_idx;
+    g.dev_status = dev_status;
+    g.idx_offset = rank * desc->vocab;
+    int used = 0;
+    if (launch_lm_head(g, reinterpret_cast<cudaStream_t>(stream), &used) != cudaSuccess) return MASSV_ERR_CUDA;
+    *n_partials = used;
+    return MASSV_OK;
+}
+
+static ShardParams shard_params(const massv_accept_desc* desc, int32_t world, int32_t rank, int32_t* dev_status) {
+    ShardParams p{};
+    p.B = desc->batch; p.gamma = desc->gamma; p.Vs = desc->vocab; p.vocab_offset = rank * desc->vocab;
+    p.T = desc->temperature; p.world = world; p.rank = rank;
+    p.n_chunks = (desc->vocab + kResidualChunk - 1) / kResidualChunk;
+    p.dev_status = dev_status;
+    return p;
+}
+
+int massv_shard_gather_draft(const massv_accept_desc* desc, int32_t world, int32_t rank, const float* logits_shard,
+                             const float* draft_probs_shard, const int32_t* draft_tokens, float* z_at_draft,
+                             float* q_at_draft, int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_shard(desc, world, rank);
+    if (rc != MASSV_OK) return rc;
+    if (desc->gamma == 0) return MASSV_OK;
+    if (!logits_shard || !draft_probs_shard || !draft_tokens || !z_at_draft || !q_at_draft) return MASSV_ERR_INVALID_ARG;
+    ShardParams p = shard_params(desc, world, rank, dev_status);
+    p.logits = logits_shard; p.draft_probs = draft_probs_shard; p.draft_tokens = draft_tokens;
+    p.z_at_draft = z_at_draft; p.q_at_draft = q_at_draft;
+    return launch_shard_gather_draft(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
+int massv_shard_scan(const massv_accept_desc* desc, int32_t world, int32_t n_partials_all, const float* part_max_all,
+                     const float* part_sum_all, const int32_t* part_idx_all, const int32_t* draft_tokens,
+                     const float* z_at_draft, const float* q_at_draft, const float* u_accept, int32_t* out_tokens,
+                     int32_t* accept_len, void* state, int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_shard(desc, world, 0);
+    if (rc != MASSV_OK) return rc;
+    const bool sampling = desc->temperature > 0.f;
+    if (n_partials_all < 1 || !part_max_all || !part_sum_all || !part_idx_all || !out_tokens || !accept_len || !state)
+        return MASSV_ERR_INVALID_ARG;
+    if (desc->gamma > 0 && (!draft_tokens || (sampling && (!z_at_draft || !q_at_draft || !u_accept))))
+        return MASSV_ERR_INVALID_ARG;
+    AcceptParams a{};
+    a.B = desc->batch; a.gamma = desc->gamma; a.V = world * desc->vocab; a.T = desc->temperature;
+    a.n_part = n_partials_all;
+    a.part_max = const_cast<float*>(part_max_all); a.part_sum = const_cast<float*>(part_sum_all);
+    a.part_idx = const_cast<int32_t*>(part_idx_all);
+    a.draft_tokens = draft_tokens; a.u_accept = u_accept;
+    a.z_at_draft = sampling ? z_at_draft : nullptr; a.q_at_draft = sampling ? q_at_draft : nullptr;
+    a.out_tokens = out_tokens; a.accept_len = accept_len;
+    a.seq_state = static_cast<SeqState*>(state);
+    a.dev_status = dev_status;
+    return launch_accept_scan_only(a, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
+int massv_shard_masses(const massv_accept_desc* desc, int32_t world, int32_t rank, const float* logits_shard,
+                       const float* draft_probs_shard, const void* state, double* mass_residual, double* mass_p,
+                       int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_shard(desc, world, rank);
+    if (rc != MASSV_OK) return rc;
+    if (!(desc->temperature > 0.f)) return MASSV_ERR_INVALID_ARG;
+    if (!logits_shard || !state || !mass_residual || !mass_p || (desc->gamma > 0 && !draft_probs_shard))
+        return MASSV_ERR_INVALID_ARG;
+    ShardParams p = shard_params(desc, world, rank, dev_status);
+    p.logits = logits_shard; p.draft_probs = draft_probs_shard; p.seq_state = static_cast<const SeqState*>(state);
+    p.sums_res = mass_residual; p.sums_p = mass_p;
+    return launch_shard_masses(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
+int massv_shard_pick(const massv_accept_desc* desc, int32_t world, int32_t rank, const double* mass_residual_all,
+                     const double* mass_p_all, const float* u_sample, const void* state, const float* logits_shard,
+                     const float* draft_probs_shard, int32_t* token_out, int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_shard(desc, world, rank);
+    if (rc != MASSV_OK) return rc;
+    if (!(desc->temperature > 0.f)) return MASSV_ERR_INVALID_ARG;
+    if (!mass_residual_all || !mass_p_all || !u_sample || !state || !logits_shard || !token_out ||
+        (desc->gamma > 0 && !draft_probs_shard))
+        return MASSV_ERR_INVALID_ARG;
+    ShardParams p = shard_params(desc, world, rank, dev_status);
+    if ((long)world * p.n_chunks > 512) return MASSV_ERR_UNSUPPORTED;
+    p.logits = logits_shard; p.draft_probs = draft_probs_shard; p.seq_state = static_cast<const SeqState*>(state);
+    p.all_res = mass_residual_all; p.all_p = mass_p_all; p.u_sample = u_sample; p.token_out = token_out;
+    return launch_shard_pick(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
+int massv_shard_set_token(const massv_accept_desc* desc, const void* state, const int32_t* tokens, int32_t* out_tokens,
+                          int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_accept_desc(desc);
+    if (rc != MASSV_OK) return rc;
+    if (!state || !tokens || !out_tokens) return MASSV_ERR_INVALID_ARG;
+    ShardParams p = shard_params(desc, 1, 0, dev_status);
+    p.seq_state = static_cast<const SeqState*>(state); p.tokens_in = tokens; p.out_tokens = out_tokens;
+    return launch_shard_set_token(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
 size_t massv_tvd_workspace_size(const massv_accept_desc* desc) {
     if (check_accept_desc(desc) != MASSV_OK || desc->gamma < 1 || !(desc->temperature > 0.f)) return 0;
     const size_t rows = (size_t)desc->batch * desc->gamma;

@@ -55,6 +55,7 @@ struct LmHeadParams {
     float *part_max, *part_sum;     // [n_part, M]
     int32_t* part_idx;              // [n_part, M]
     int32_t* dev_status;
+    int idx_offset = 0;             // added to the argmax indices (first vocabulary row of a shard)
 };
 int lm_head_num_partials(int M, int V);            // upper bound of the partial slots, for workspace sizing
 // *n_part_used receives the number of slots this launch fills (<= p.n_part).
@@ -77,8 +78,39 @@ struct AcceptParams {
     unsigned int* counters;         // [B]
     int n_chunks;
     int32_t* dev_status;
+    // vocabulary-sharded use: the target's logit and the drafter's probability at every drafted token,
+    // collected from the rank that owns the token (then `logits` / `draft_probs` are not read by the scan)
+    const float* z_at_draft = nullptr;   // [B, gamma]
+    const float* q_at_draft = nullptr;   // [B, gamma]
 };
 cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream);
+cudaError_t launch_accept_scan_only(const AcceptParams& p, cudaStream_t stream);
+
+// ---------------------------------------------------------------- vocabulary shards
+struct ShardParams {
+    int B, gamma, Vs;               // Vs: vocabulary entries of this shard
+    int vocab_offset;               // first vocabulary index of this shard
+    float T;
+    const float* logits;            // [B*(gamma+1), Vs]
+    const float* draft_probs;       // [B, gamma, Vs]
+    const int32_t* draft_tokens;    // [B, gamma]
+    float *z_at_draft, *q_at_draft; // [B, gamma]: -inf where another shard owns the token
+    const SeqState* seq_state;      // [B]
+    double *sums_res, *sums_p;      // [B, n_chunks]: chunk masses of max(p - q, 0) and of p on the sampled row
+    int n_chunks;                   // chunks of this shard
+    // pick
+    const double *all_res, *all_p;  // [world, B, n_chunks]: ranks in order are vocabulary order
+    int world, rank;
+    const float* u_sample;          // [B, gamma+1]
+    int32_t* token_out;             // [B]: the drawn token if this shard owns it, else -1
+    int32_t* out_tokens;            // [B, gamma+1]
+    const int32_t* tokens_in;       // [B]
+    int32_t* dev_status;
+};
+cudaError_t launch_shard_gather_draft(const ShardParams& p, cudaStream_t stream);
+cudaError_t launch_shard_masses(const ShardParams& p, cudaStream_t stream);
+cudaError_t launch_shard_pick(const ShardParams& p, cudaStream_t stream);
+cudaError_t launch_shard_set_token(const ShardParams& p, cudaStream_t stream);
 
 // ---------------------------------------------------------------- TVD diagnostic
 constexpr int kTvdSlices = 16;      // vocabulary slices per row

@@ -49,6 +49,7 @@ struct UmmaParams {
     float *part_max, *part_sum;
     int32_t* part_idx;
     int32_t* dev_status;
+    int idx_offset;      // added to the argmax indices that leave the kernel
 };
 
 // ---- CTA pairs (cta_group::2): two CTAs of a cluster act as one 256-row MMA.  Each loads its own
@@ -460,7 +461,7 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             const size_t slot = (size_t)(PAIR ? group * 2 + (int)pair_rank : group) * p.M;
             p.part_max[slot + tok] = acc.m;
             p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
-            p.part_idx[slot + tok] = acc.idx;
+            p.part_idx[slot + tok] = acc.idx == 0x7fffffff ? acc.idx : acc.idx + p.idx_offset;
         }
     }
     if constexpr (PAIR) cluster_sync_all();      // neither CTA frees TMEM or leaves while the other may still use it
@@ -528,6 +529,7 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.logits = q.logits;
     p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
     p.dev_status = q.dev_status;
+    p.idx_offset = q.idx_offset;
     const int slots = groups * (pair ? 2 : 1);
     if (slots > q.n_part) return cudaErrorInvalidValue;
     *n_part_used = slots;

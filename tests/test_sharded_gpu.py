@@ -1,0 +1,101 @@
+"""Vocabulary-sharded acceptance vs the CPU oracle of the unsharded step.
+
+All ranks of a world run on ONE device, phase by phase (``run_lockstep``): every rank's kernels finish
+before the exchange that follows them, so no kernel waits on another.  The oracle never sees a shard: it
+computes the whole-vocabulary step, and the sharded result must agree with it exactly as the unsharded
+kernel path does (bit-exact tokens and lengths, except at decisions whose oracle margin is below 1e-3).
+"""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from parity_util import compare_accept, sub_workload
+from workloads import generate, get_config
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_sharded(cfg, w, world):
+    from paper_2505_10526_b200.sharded import ShardedAccept, run_lockstep
+    assert cfg.vocab % world == 0
+    Vs = cfg.vocab // world
+    ranks = [ShardedAccept(cfg.batch, cfg.gamma, cfg.hidden, Vs, cfg.temperature, world, r) for r in range(world)]
+    inputs = []
+    for r in range(world):
+        kw = dict(hidden=w["hidden"], lm_head_shard=w["lm_head"][r * Vs:(r + 1) * Vs].contiguous(),
+                  draft_tokens=w["draft_tokens"])
+        if cfg.temperature > 0:
+            kw.update(draft_probs_shard=w["draft_probs"][:, :, r * Vs:(r + 1) * Vs].contiguous(),
+                      u_accept=w["u_accept"], u_sample=w["u_sample"])
+        inputs.append(kw)
+    res = run_lockstep(ranks, inputs)
+    torch.cuda.synchronize()
+    for rk in ranks:
+        assert int(rk.dev_status.item()) == 0
+    toks, lens = res[0]
+    for t, l in res[1:]:                       # every rank ends with the same answer
+        assert torch.equal(t, toks) and torch.equal(l, lens)
+    return toks, lens, ranks
+
+
+def _check(cfg, world, subset=None, w=None):
+    w = w or generate(cfg, device="cuda", with_attention=False)
+    toks, lens, ranks = _run_sharded(cfg, w, world)
+    idx = list(range(cfg.batch)) if subset is None else subset
+    ref = oracle.verify_step(sub_workload(w, idx), cfg.temperature, want_attention=False)
+    sel = torch.as_tensor(idx, device="cuda")
+    st = compare_accept(ref, toks.index_select(0, sel).cpu().numpy(), lens.index_select(0, sel).cpu().numpy(), cfg.gamma)
+    print(dict(config=cfg.name, world=world, **{k: v for k, v in st.items() if k != "details"}))
+    assert st["hard"] == 0, st["details"]
+    if cfg.temperature > 0:                    # the shards' logits are the oracle's columns
+        R, V, Vs = cfg.rows, cfg.vocab, cfg.vocab // world
+        z = torch.cat([rk.logits for rk in ranks], dim=1).view(cfg.batch, R, V).index_select(0, sel)
+        assert float(np.abs(z.cpu().double().numpy().reshape(-1, V) - ref["logits"]).max()) < 2e-2
+    return toks, lens
+
+
+@pytest.mark.parametrize("world", [1, 2, 4])
+@pytest.mark.parametrize("name", ["tiny_t0", "tiny_t1", "tiny_ragged_t0", "tiny_ragged_t1", "tiny_peaked_t1"])
+def test_tiny_configs(name, world):
+    _check(get_config(name), world)
+
+
+@pytest.mark.parametrize("world", [2, 5])
+@pytest.mark.parametrize("t", [0.0, 0.8])
+def test_shards_of_several_chunks_with_a_ragged_last_chunk(world, t):
+    """20480 * 5 / world entries per shard: 3 to 13 chunks of 4096, the last one partial."""
+    cfg = replace(get_config("tiny_ragged_t1"), name=f"chunks_w{world}", vocab=20480 * 5, temperature=t, batch=6, seed=77)
+    _check(cfg, world)
+
+
+def test_sharded_result_equals_the_unsharded_call():
+    """Same inputs through massv_accept and through four shards: identical tokens and lengths."""
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = replace(get_config("tiny_peaked_t1"), vocab=32768, batch=8, seed=5)
+    w = generate(cfg, device="cuda")
+    toks, lens, _ = _run_sharded(cfg, w, 4)
+    step = VerifyStep.for_workload(cfg, w)
+    step.run(w, commit=False)
+    torch.cuda.synchronize()
+    assert torch.equal(step.accept_len, lens)
+    assert torch.equal(step.out_tokens, toks)
+
+
+def test_every_draft_accepted_draws_the_bonus_token_across_shards():
+    """Uniforms of 0 accept every drafted token whose p is positive, so the extra token is the bonus draw
+    from p itself (no residual): the walk over the shards' chunk masses of p picks it."""
+    cfg = replace(get_config("tiny_t1"), batch=3, seed=9)
+    w = generate(cfg, device="cuda", with_attention=False)
+    w["u_accept"].zero_()
+    toks, lens = _check(cfg, 2, w=w)
+    assert bool((lens == cfg.gamma + 1).all())
+
+
+@pytest.mark.parametrize("name,world,subset", [("qwen7b_b1_t0", 2, None), ("qwen7b_b16_t1", 4, [0, 7, 15]),
+                                               ("qwen7b_b16_t1_peaked", 8, [3, 12])])
+def test_full_size_vocabulary(name, world, subset):
+    cfg = get_config(name)
+    _check(cfg, world, subset=subset)
