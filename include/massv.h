@@ -268,58 +268,59 @@ int massv_sample_top_p(int32_t rows, int32_t vocab, float temperature, float top
  * prefix rule at temperature 0); only where the data lives changes.  Rank r holds rows
  * [r * vocab, (r + 1) * vocab) of the LM head and the same columns of q: desc->vocab is the SHARD's size,
  * equal on every rank, so the whole vocabulary is world * vocab.  The library exchanges nothing itself:
- * between the calls the caller all-gathers three small buffers (NCCL or any other transport), and every
- * rank then takes the same decisions from the same gathered values.  Per step, on every rank:
+ * each rank fills an exchange buffer, the caller all-gathers it (NCCL or any other transport; rank r's
+ * copy at offset r * size of the gathered buffer), and every rank then takes the same decisions from the
+ * same gathered values.  Three all-gathers per step at T > 0, one at T == 0.  On every rank:
  *
- *   1. massv_shard_lm_head      logits of the shard (+ per-row max / sum-exp / argmax partials, argmax
- *                               indices already global); *n_partials (host) = slots written.
- *   2. massv_shard_gather_draft (T > 0) logit and q at each drafted token this rank owns, -inf elsewhere;
- *                               the caller reduces both with MAX over the ranks.
- *      all-gather the first n_partials slots of part_max / part_sum / part_idx along the slot axis.
- *   3. massv_shard_scan         merges the partials of all ranks, runs the rejection test (or the greedy
- *                               prefix rule), writes accept_len, the accepted drafts into out_tokens and,
- *                               at T == 0, the extra token; fills `state` (massv_shard_state_bytes).
- *                               T == 0 ends here.
+ *   1. massv_shard_lm_head      logits of the shard; per-row max / sum-exp / argmax partials (argmax
+ *                               indices already global) go into `stats`; *n_partials (host) = partial
+ *                               slots written, the same on every rank.
+ *   2. massv_shard_gather_draft (T > 0) logit and q at each drafted token this rank owns, -inf
+ *                               elsewhere, into `stats`.
+ *      all-gather `stats`: fp32 words, massv_shard_stats_words per rank.
+ *   3. massv_shard_scan         merges the partials of all ranks (ranks in order), takes the owner's
+ *                               values at the drafted tokens, runs the rejection test (or the greedy
+ *                               prefix rule), writes accept_len, the accepted drafts into out_tokens
+ *                               and, at T == 0, the extra token; fills `state`
+ *                               (massv_shard_state_bytes).  T == 0 ends here.
  *   4. massv_shard_masses       masses of this shard's 4096-entry chunks of the row the extra token is
  *                               drawn from: of max(p - q, 0) (of p for the bonus row) and of p.
- *      all-gather both arrays: [world, batch, massv_shard_chunks].
+ *      all-gather `masses`: fp64, massv_shard_mass_count per rank.
  *   5. massv_shard_pick         every rank walks the gathered masses (ranks in order = vocabulary
  *                               order) to the chunk where the running mass passes u * total; the rank
  *                               that owns it stores the token (global index), the others -1.  A
  *                               residual without mass anywhere falls back to p, as massv_accept does.
- *      reduce token_out with MAX over the ranks.
- *   6. massv_shard_set_token    stores the agreed token at out_tokens[b, accept_len[b] - 1].
+ *      all-gather token_out: int32 [batch] per rank.
+ *   6. massv_shard_set_token    stores the owner's token at out_tokens[b, accept_len[b] - 1].
  *
- * Shapes: part_* [massv_shard_max_partials, batch * (gamma + 1)] per rank; z_at_draft, q_at_draft
- * fp32 [batch, gamma]; mass_* fp64 [batch, massv_shard_chunks]; token_out / tokens int32 [batch];
  * logits_shard fp32 [batch * (gamma + 1), vocab] (required at T > 0, optional at T == 0);
- * draft_probs_shard fp32 [batch, gamma, vocab].  world * massv_shard_chunks <= 512.  All pointers are
- * device pointers except n_partials.  Errors as for massv_accept.
+ * draft_probs_shard fp32 [batch, gamma, vocab]; u_accept, u_sample, draft_tokens, out_tokens,
+ * accept_len as for massv_accept.  world * ceil(vocab / 4096) <= 512.  `stats` 16-byte aligned.  All
+ * pointers are device pointers except n_partials.  Errors as for massv_accept.
  */
-size_t massv_shard_max_partials(const massv_accept_desc *desc);
-size_t massv_shard_chunks(const massv_accept_desc *desc);
+size_t massv_shard_stats_words(const massv_accept_desc *desc);
+size_t massv_shard_mass_count(const massv_accept_desc *desc);
 size_t massv_shard_state_bytes(const massv_accept_desc *desc);
 int massv_shard_lm_head(const massv_accept_desc *desc, int32_t world, int32_t rank, const void *hidden,
-                        const void *lm_head_shard, float *logits_shard, float *part_max, float *part_sum,
-                        int32_t *part_idx, int32_t *n_partials, int32_t *dev_status, massv_stream_t stream);
+                        const void *lm_head_shard, float *logits_shard, float *stats, int32_t *n_partials,
+                        int32_t *dev_status, massv_stream_t stream);
 int massv_shard_gather_draft(const massv_accept_desc *desc, int32_t world, int32_t rank,
                              const float *logits_shard, const float *draft_probs_shard,
-                             const int32_t *draft_tokens, float *z_at_draft, float *q_at_draft,
-                             int32_t *dev_status, massv_stream_t stream);
-int massv_shard_scan(const massv_accept_desc *desc, int32_t world, int32_t n_partials_all,
-                     const float *part_max_all, const float *part_sum_all, const int32_t *part_idx_all,
-                     const int32_t *draft_tokens, const float *z_at_draft, const float *q_at_draft,
-                     const float *u_accept, int32_t *out_tokens, int32_t *accept_len, void *state,
-                     int32_t *dev_status, massv_stream_t stream);
+                             const int32_t *draft_tokens, float *stats, int32_t *dev_status,
+                             massv_stream_t stream);
+int massv_shard_scan(const massv_accept_desc *desc, int32_t world, int32_t n_partials, const float *stats_all,
+                     const int32_t *draft_tokens, const float *u_accept, int32_t *out_tokens,
+                     int32_t *accept_len, void *state, int32_t *dev_status, massv_stream_t stream);
 int massv_shard_masses(const massv_accept_desc *desc, int32_t world, int32_t rank, const float *logits_shard,
-                       const float *draft_probs_shard, const void *state, double *mass_residual,
-                       double *mass_p, int32_t *dev_status, massv_stream_t stream);
-int massv_shard_pick(const massv_accept_desc *desc, int32_t world, int32_t rank,
-                     const double *mass_residual_all, const double *mass_p_all, const float *u_sample,
-                     const void *state, const float *logits_shard, const float *draft_probs_shard,
-                     int32_t *token_out, int32_t *dev_status, massv_stream_t stream);
-int massv_shard_set_token(const massv_accept_desc *desc, const void *state, const int32_t *tokens,
-                          int32_t *out_tokens, int32_t *dev_status, massv_stream_t stream);
+                       const float *draft_probs_shard, const void *state, double *masses,
+                       int32_t *dev_status, massv_stream_t stream);
+int massv_shard_pick(const massv_accept_desc *desc, int32_t world, int32_t rank, const double *masses_all,
+                     const float *u_sample, const void *state, const float *logits_shard,
+                     const float *draft_probs_shard, int32_t *token_out, int32_t *dev_status,
+                     massv_stream_t stream);
+int massv_shard_set_token(const massv_accept_desc *desc, int32_t world, const void *state,
+                          const int32_t *tokens_all, int32_t *out_tokens, int32_t *dev_status,
+                          massv_stream_t stream);
 
 /* Human-readable name of a massv_status value. */
 const char *massv_strerror(int status);

@@ -60,22 +60,22 @@ def _load():
     lib.massv_tvd.argtypes = [ctypes.POINTER(AcceptDesc), f32p, f32p, f32p, f32p, vp, ctypes.c_size_t, i32p, vp]
     lib.massv_sample_top_p.restype = ctypes.c_int
     lib.massv_sample_top_p.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_float, f32p, f32p, i32p, f32p, i32p, vp]
-    D, i32, f64p = ctypes.POINTER(AcceptDesc), ctypes.c_int32, vp
-    for name in ("massv_shard_max_partials", "massv_shard_chunks", "massv_shard_state_bytes"):
+    D, i32 = ctypes.POINTER(AcceptDesc), ctypes.c_int32
+    for name in ("massv_shard_stats_words", "massv_shard_mass_count", "massv_shard_state_bytes"):
         getattr(lib, name).restype = ctypes.c_size_t
         getattr(lib, name).argtypes = [D]
     lib.massv_shard_lm_head.restype = ctypes.c_int
-    lib.massv_shard_lm_head.argtypes = [D, i32, i32, vp, vp, f32p, f32p, f32p, i32p, ctypes.POINTER(ctypes.c_int32), i32p, vp]
+    lib.massv_shard_lm_head.argtypes = [D, i32, i32, vp, vp, f32p, f32p, ctypes.POINTER(ctypes.c_int32), i32p, vp]
     lib.massv_shard_gather_draft.restype = ctypes.c_int
-    lib.massv_shard_gather_draft.argtypes = [D, i32, i32, f32p, f32p, i32p, f32p, f32p, i32p, vp]
+    lib.massv_shard_gather_draft.argtypes = [D, i32, i32, f32p, f32p, i32p, f32p, i32p, vp]
     lib.massv_shard_scan.restype = ctypes.c_int
-    lib.massv_shard_scan.argtypes = [D, i32, i32, f32p, f32p, i32p, i32p, f32p, f32p, f32p, i32p, i32p, vp, i32p, vp]
+    lib.massv_shard_scan.argtypes = [D, i32, i32, f32p, i32p, f32p, i32p, i32p, vp, i32p, vp]
     lib.massv_shard_masses.restype = ctypes.c_int
-    lib.massv_shard_masses.argtypes = [D, i32, i32, f32p, f32p, vp, f64p, f64p, i32p, vp]
+    lib.massv_shard_masses.argtypes = [D, i32, i32, f32p, f32p, vp, vp, i32p, vp]
     lib.massv_shard_pick.restype = ctypes.c_int
-    lib.massv_shard_pick.argtypes = [D, i32, i32, f64p, f64p, f32p, vp, f32p, f32p, i32p, i32p, vp]
+    lib.massv_shard_pick.argtypes = [D, i32, i32, vp, f32p, vp, f32p, f32p, i32p, i32p, vp]
     lib.massv_shard_set_token.restype = ctypes.c_int
-    lib.massv_shard_set_token.argtypes = [D, vp, i32p, i32p, i32p, vp]
+    lib.massv_shard_set_token.argtypes = [D, i32, vp, i32p, i32p, i32p, vp]
     lib.massv_kv_commit.restype = ctypes.c_int
     lib.massv_kv_commit.argtypes = [ctypes.c_int32, ctypes.c_int32, i32p, i32p, i32p, vp]
     lib.massv_strerror.restype = ctypes.c_char_p
@@ -226,12 +226,12 @@ def massv_sample_top_p(logits, u, tokens, temperature, top_p, probs_out=None, de
 
 
 # ---- vocabulary shards (argument marshalling only; the caller moves the gathered buffers between ranks)
-def massv_shard_max_partials(desc) -> int:
-    return int(_lib.massv_shard_max_partials(ctypes.byref(desc)))
+def massv_shard_stats_words(desc) -> int:
+    return int(_lib.massv_shard_stats_words(ctypes.byref(desc)))
 
 
-def massv_shard_chunks(desc) -> int:
-    return int(_lib.massv_shard_chunks(ctypes.byref(desc)))
+def massv_shard_mass_count(desc) -> int:
+    return int(_lib.massv_shard_mass_count(ctypes.byref(desc)))
 
 
 def massv_shard_state_bytes(desc) -> int:
@@ -243,57 +243,50 @@ def _check(rc, name):
         raise MassvError(rc, name)
 
 
-def massv_shard_lm_head(desc, world, rank, hidden, lm_head_shard, logits_shard, part_max, part_sum, part_idx,
-                        dev_status=None) -> int:
+def massv_shard_lm_head(desc, world, rank, hidden, lm_head_shard, logits_shard, stats, dev_status=None) -> int:
     """Returns the number of partial slots written (the same on every rank)."""
     bf, f32, i32 = torch.bfloat16, torch.float32, torch.int32
     n = ctypes.c_int32(0)
     _check(_lib.massv_shard_lm_head(ctypes.byref(desc), world, rank, _ptr(hidden, bf), _ptr(lm_head_shard, bf),
-                                    _ptr(logits_shard, f32), _ptr(part_max, f32), _ptr(part_sum, f32),
-                                    _ptr(part_idx, i32), ctypes.byref(n), _ptr(dev_status, i32), _stream()),
-           "massv_shard_lm_head")
+                                    _ptr(logits_shard, f32), _ptr(stats, f32), ctypes.byref(n), _ptr(dev_status, i32),
+                                    _stream()), "massv_shard_lm_head")
     return int(n.value)
 
 
-def massv_shard_gather_draft(desc, world, rank, logits_shard, draft_probs_shard, draft_tokens, z_at_draft, q_at_draft,
+def massv_shard_gather_draft(desc, world, rank, logits_shard, draft_probs_shard, draft_tokens, stats,
                              dev_status=None) -> None:
     f32, i32 = torch.float32, torch.int32
     _check(_lib.massv_shard_gather_draft(ctypes.byref(desc), world, rank, _ptr(logits_shard, f32),
-                                         _ptr(draft_probs_shard, f32), _ptr(draft_tokens, i32), _ptr(z_at_draft, f32),
-                                         _ptr(q_at_draft, f32), _ptr(dev_status, i32), _stream()),
-           "massv_shard_gather_draft")
+                                         _ptr(draft_probs_shard, f32), _ptr(draft_tokens, i32), _ptr(stats, f32),
+                                         _ptr(dev_status, i32), _stream()), "massv_shard_gather_draft")
 
 
-def massv_shard_scan(desc, world, n_partials_all, part_max_all, part_sum_all, part_idx_all, draft_tokens, z_at_draft,
-                     q_at_draft, u_accept, out_tokens, accept_len, state, dev_status=None) -> None:
+def massv_shard_scan(desc, world, n_partials, stats_all, draft_tokens, u_accept, out_tokens, accept_len, state,
+                     dev_status=None) -> None:
     f32, i32 = torch.float32, torch.int32
-    _check(_lib.massv_shard_scan(ctypes.byref(desc), world, n_partials_all, _ptr(part_max_all, f32),
-                                 _ptr(part_sum_all, f32), _ptr(part_idx_all, i32), _ptr(draft_tokens, i32),
-                                 _ptr(z_at_draft, f32), _ptr(q_at_draft, f32), _ptr(u_accept, f32),
-                                 _ptr(out_tokens, i32), _ptr(accept_len, i32), _ptr(state, torch.uint8),
-                                 _ptr(dev_status, i32), _stream()), "massv_shard_scan")
+    _check(_lib.massv_shard_scan(ctypes.byref(desc), world, n_partials, _ptr(stats_all, f32), _ptr(draft_tokens, i32),
+                                 _ptr(u_accept, f32), _ptr(out_tokens, i32), _ptr(accept_len, i32),
+                                 _ptr(state, torch.uint8), _ptr(dev_status, i32), _stream()), "massv_shard_scan")
 
 
-def massv_shard_masses(desc, world, rank, logits_shard, draft_probs_shard, state, mass_residual, mass_p,
-                       dev_status=None) -> None:
+def massv_shard_masses(desc, world, rank, logits_shard, draft_probs_shard, state, masses, dev_status=None) -> None:
     f32, f64, i32 = torch.float32, torch.float64, torch.int32
     _check(_lib.massv_shard_masses(ctypes.byref(desc), world, rank, _ptr(logits_shard, f32),
-                                   _ptr(draft_probs_shard, f32), _ptr(state, torch.uint8), _ptr(mass_residual, f64),
-                                   _ptr(mass_p, f64), _ptr(dev_status, i32), _stream()), "massv_shard_masses")
+                                   _ptr(draft_probs_shard, f32), _ptr(state, torch.uint8), _ptr(masses, f64),
+                                   _ptr(dev_status, i32), _stream()), "massv_shard_masses")
 
 
-def massv_shard_pick(desc, world, rank, mass_residual_all, mass_p_all, u_sample, state, logits_shard,
-                     draft_probs_shard, token_out, dev_status=None) -> None:
+def massv_shard_pick(desc, world, rank, masses_all, u_sample, state, logits_shard, draft_probs_shard, token_out,
+                     dev_status=None) -> None:
     f32, f64, i32 = torch.float32, torch.float64, torch.int32
-    _check(_lib.massv_shard_pick(ctypes.byref(desc), world, rank, _ptr(mass_residual_all, f64), _ptr(mass_p_all, f64),
-                                 _ptr(u_sample, f32), _ptr(state, torch.uint8), _ptr(logits_shard, f32),
-                                 _ptr(draft_probs_shard, f32), _ptr(token_out, i32), _ptr(dev_status, i32), _stream()),
-           "massv_shard_pick")
+    _check(_lib.massv_shard_pick(ctypes.byref(desc), world, rank, _ptr(masses_all, f64), _ptr(u_sample, f32),
+                                 _ptr(state, torch.uint8), _ptr(logits_shard, f32), _ptr(draft_probs_shard, f32),
+                                 _ptr(token_out, i32), _ptr(dev_status, i32), _stream()), "massv_shard_pick")
 
 
-def massv_shard_set_token(desc, state, tokens, out_tokens, dev_status=None) -> None:
+def massv_shard_set_token(desc, world, state, tokens_all, out_tokens, dev_status=None) -> None:
     i32 = torch.int32
-    _check(_lib.massv_shard_set_token(ctypes.byref(desc), _ptr(state, torch.uint8), _ptr(tokens, i32),
+    _check(_lib.massv_shard_set_token(ctypes.byref(desc), world, _ptr(state, torch.uint8), _ptr(tokens_all, i32),
                                       _ptr(out_tokens, i32), _ptr(dev_status, i32), _stream()), "massv_shard_set_token")
 
 

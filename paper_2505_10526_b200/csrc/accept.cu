@@ -63,9 +63,12 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
                 const int i = i0 + k * 32 + lane;
                 x[k] = Stat{-INFINITY, 0.f, 0x7fffffff};
                 if (i < p.n_part) {
-                    x[k].m = p.part_max[(size_t)i * M + row];
-                    x[k].s = greedy ? 0.f : p.part_sum[(size_t)i * M + row];
-                    x[k].idx = p.part_idx[(size_t)i * M + row];
+                    const size_t at = p.part_per_rank
+                        ? (size_t)(i / p.part_per_rank) * p.rank_stride + (size_t)(i % p.part_per_rank) * M + row
+                        : (size_t)i * M + row;
+                    x[k].m = p.part_max[at];
+                    x[k].s = greedy ? 0.f : p.part_sum[at];
+                    x[k].idx = p.part_idx[at];
                 }
             }
 #pragma unroll
@@ -95,9 +98,18 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
         } else if (greedy) {
             ok = (x == row_stat[lane].idx);
         } else {
-            const float zx = p.z_at_draft ? p.z_at_draft[(size_t)b * p.gamma + lane] : p.logits[(size_t)(b * R + lane) * p.V + x];
+            float zx, qx;
+            if (p.z_at_draft) {                 // the owner's value is the only one that is not -inf
+                zx = qx = -INFINITY;
+                for (int r = 0; r < p.ranks; ++r) {
+                    zx = fmaxf(zx, p.z_at_draft[r * p.rank_stride + (size_t)b * p.gamma + lane]);
+                    qx = fmaxf(qx, p.q_at_draft[r * p.rank_stride + (size_t)b * p.gamma + lane]);
+                }
+            } else {
+                zx = p.logits[(size_t)(b * R + lane) * p.V + x];
+                qx = p.draft_probs[((size_t)b * p.gamma + lane) * p.V + x];
+            }
             const float px = expf((zx - row_stat[lane].m) * inv_T) / row_stat[lane].s;
-            const float qx = p.q_at_draft ? p.q_at_draft[(size_t)b * p.gamma + lane] : p.draft_probs[((size_t)b * p.gamma + lane) * p.V + x];
             const float lhs = p.u_accept[(size_t)b * p.gamma + lane] * qx;
             ok = lhs < px;
         }
@@ -369,10 +381,10 @@ __global__ void __launch_bounds__(kSampleThreads) shard_pick_kernel(ShardParams 
     }
     int use_q = st.use_q;
     for (int attempt = 0; attempt < 2; ++attempt) {
-        // gathered layout [world, B, n_chunks]: rank r's chunks of sequence b are contiguous
+        // rank r's chunks of sequence b are contiguous inside r's copy of the exchange buffer
         const double* sums = use_q ? p.all_res : p.all_p;
         for (int i = t; i < n_all; i += kSampleThreads)
-            s_sums[i] = sums[((size_t)(i / p.n_chunks) * p.B + b) * p.n_chunks + i % p.n_chunks];
+            s_sums[i] = sums[(size_t)(i / p.n_chunks) * p.mass_rank_stride + (size_t)b * p.n_chunks + i % p.n_chunks];
         __syncthreads();
         if (t == 0) {
             double tot = 0.0;
@@ -438,7 +450,8 @@ __global__ void shard_set_token_kernel(ShardParams p) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait();
     if (b >= p.B) return;
-    const int tok = p.tokens_in[b];
+    int tok = -1;
+    for (int r = 0; r < p.world; ++r) tok = max(tok, p.tokens_in[(size_t)r * p.B + b]);
     if (tok < 0) { set_status(p.dev_status, MASSV_ERR_INVALID_ARG); return; }
     p.out_tokens[(size_t)b * (p.gamma + 1) + p.seq_state[b].n] = tok;
 }

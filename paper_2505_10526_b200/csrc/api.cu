@@ -212,15 +212,56 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
     return launch_accept(a, s) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
+}  // extern "C"
+
 // ---------------------------------------------------------------- vocabulary shards
-size_t massv_shard_max_partials(const massv_accept_desc* desc) {
-    if (check_accept_desc(desc) != MASSV_OK) return 0;
-    return (size_t)lm_head_num_partials(desc->batch * (desc->gamma + 1), desc->vocab);
+namespace {
+// Exchange buffer A of one rank, in 4-byte words: the three partial arrays, then z and q at the drafted tokens.
+struct ShardLayoutA {
+    int slots;
+    size_t M, off_max, off_sum, off_idx, off_z, off_q, words;
+};
+ShardLayoutA shard_layout_a(const massv_accept_desc& d) {
+    ShardLayoutA l;
+    l.M = (size_t)d.batch * (d.gamma + 1);
+    l.slots = lm_head_num_partials((int)l.M, d.vocab);
+    const size_t part = (size_t)l.slots * l.M, at = (size_t)d.batch * d.gamma;
+    l.off_max = 0; l.off_sum = part; l.off_idx = 2 * part; l.off_z = 3 * part; l.off_q = 3 * part + at;
+    l.words = (3 * part + 2 * at + 3) & ~(size_t)3;          // every rank's copy starts 16-byte aligned
+    return l;
+}
+int shard_chunks(const massv_accept_desc& d) { return (d.vocab + kResidualChunk - 1) / kResidualChunk; }
+
+int check_shard(const massv_accept_desc* desc, int32_t world, int32_t rank) {
+    const int rc = check_accept_desc(desc);
+    if (rc != MASSV_OK) return rc;
+    if (world < 1 || rank < 0 || rank >= world) return MASSV_ERR_INVALID_ARG;
+    if ((long)world * desc->vocab > 0x7fffffffL) return MASSV_ERR_UNSUPPORTED;
+    if ((long)world * shard_chunks(*desc) > 512) return MASSV_ERR_UNSUPPORTED;
+    return MASSV_OK;
 }
 
-size_t massv_shard_chunks(const massv_accept_desc* desc) {
+ShardParams shard_params(const massv_accept_desc* desc, int32_t world, int32_t rank, int32_t* dev_status) {
+    ShardParams p{};
+    p.B = desc->batch; p.gamma = desc->gamma; p.Vs = desc->vocab; p.vocab_offset = rank * desc->vocab;
+    p.T = desc->temperature; p.world = world; p.rank = rank;
+    p.n_chunks = shard_chunks(*desc);
+    p.mass_rank_stride = (size_t)2 * desc->batch * p.n_chunks;
+    p.dev_status = dev_status;
+    return p;
+}
+}  // namespace
+
+extern "C" {
+
+size_t massv_shard_stats_words(const massv_accept_desc* desc) {
     if (check_accept_desc(desc) != MASSV_OK) return 0;
-    return (size_t)((desc->vocab + kResidualChunk - 1) / kResidualChunk);
+    return shard_layout_a(*desc).words;
+}
+
+size_t massv_shard_mass_count(const massv_accept_desc* desc) {
+    if (check_accept_desc(desc) != MASSV_OK) return 0;
+    return (size_t)2 * desc->batch * shard_chunks(*desc);
 }
 
 size_t massv_shard_state_bytes(const massv_accept_desc* desc) {
@@ -228,33 +269,27 @@ size_t massv_shard_state_bytes(const massv_accept_desc* desc) {
     return (size_t)desc->batch * sizeof(SeqState);
 }
 
-static int check_shard(const massv_accept_desc* desc, int32_t world, int32_t rank) {
-    const int rc = check_accept_desc(desc);
-    if (rc != MASSV_OK) return rc;
-    if (world < 1 || rank < 0 || rank >= world) return MASSV_ERR_INVALID_ARG;
-    if ((long)world * desc->vocab > 0x7fffffffL) return MASSV_ERR_UNSUPPORTED;
-    return MASSV_OK;
-}
-
 int massv_shard_lm_head(const massv_accept_desc* desc, int32_t world, int32_t rank, const void* hidden,
-                        const void* lm_head_shard, float* logits_shard, float* part_max, float* part_sum,
-                        int32_t* part_idx, int32_t* n_partials, int32_t* dev_status, massv_stream_t stream) {
+                        const void* lm_head_shard, float* logits_shard, float* stats, int32_t* n_partials,
+                        int32_t* dev_status, massv_stream_t stream) {
     const int rc = check_shard(desc, world, rank);
     if (rc != MASSV_OK) return rc;
     const bool sampling = desc->temperature > 0.f;
-    if (!hidden || !lm_head_shard || !part_max || !part_sum || !part_idx || !n_partials) return MASSV_ERR_INVALID_ARG;
+    if (!hidden || !lm_head_shard || !stats || !n_partials) return MASSV_ERR_INVALID_ARG;
     if (sampling && !logits_shard) return MASSV_ERR_INVALID_ARG;
-    if (!aligned16(hidden) || !aligned16(lm_head_shard) || (logits_shard && !aligned16(logits_shard)))
+    if (!aligned16(hidden) || !aligned16(lm_head_shard) || !aligned16(stats) || (logits_shard && !aligned16(logits_shard)))
         return MASSV_ERR_INVALID_ARG;
+    const ShardLayoutA l = shard_layout_a(*desc);
     LmHeadParams g;
-    g.M = desc->batch * (desc->gamma + 1); g.K = desc->hidden; g.V = desc->vocab;
+    g.M = (int)l.M; g.K = desc->hidden; g.V = desc->vocab;
     g.greedy = sampling ? 0 : 1;
     g.inv_T_log2e = sampling ? 1.4426950408889634f / desc->temperature : 0.f;
     g.hidden = static_cast<const __nv_bfloat16*>(hidden);
     g.lm_head = static_cast<const __nv_bfloat16*>(lm_head_shard);
     g.logits = logits_shard;
-    g.n_part = lm_head_num_partials(g.M, g.V);
-    g.part_max = part_max; g.part_sum = part_sum; g.part_idx = part_idx;
+    g.n_part = l.slots;
+    g.part_max = stats + l.off_max; g.part_sum = stats + l.off_sum;
+    g.part_idx = reinterpret_cast<int32_t*>(stats + l.off_idx);
     g.dev_status = dev_status;
     g.idx_offset = rank * desc->vocab;
     int used = 0;
@@ -263,46 +298,37 @@ int massv_shard_lm_head(const massv_accept_desc* desc, int32_t world, int32_t ra
     return MASSV_OK;
 }
 
-static ShardParams shard_params(const massv_accept_desc* desc, int32_t world, int32_t rank, int32_t* dev_status) {
-    ShardParams p{};
-    p.B = desc->batch; p.gamma = desc->gamma; p.Vs = desc->vocab; p.vocab_offset = rank * desc->vocab;
-    p.T = desc->temperature; p.world = world; p.rank = rank;
-    p.n_chunks = (desc->vocab + kResidualChunk - 1) / kResidualChunk;
-    p.dev_status = dev_status;
-    return p;
-}
-
 int massv_shard_gather_draft(const massv_accept_desc* desc, int32_t world, int32_t rank, const float* logits_shard,
-                             const float* draft_probs_shard, const int32_t* draft_tokens, float* z_at_draft,
-                             float* q_at_draft, int32_t* dev_status, massv_stream_t stream) {
+                             const float* draft_probs_shard, const int32_t* draft_tokens, float* stats,
+                             int32_t* dev_status, massv_stream_t stream) {
     const int rc = check_shard(desc, world, rank);
     if (rc != MASSV_OK) return rc;
-    if (desc->gamma == 0) return MASSV_OK;
-    if (!logits_shard || !draft_probs_shard || !draft_tokens || !z_at_draft || !q_at_draft) return MASSV_ERR_INVALID_ARG;
+    if (desc->gamma == 0 || !(desc->temperature > 0.f)) return MASSV_OK;
+    if (!logits_shard || !draft_probs_shard || !draft_tokens || !stats) return MASSV_ERR_INVALID_ARG;
+    const ShardLayoutA l = shard_layout_a(*desc);
     ShardParams p = shard_params(desc, world, rank, dev_status);
     p.logits = logits_shard; p.draft_probs = draft_probs_shard; p.draft_tokens = draft_tokens;
-    p.z_at_draft = z_at_draft; p.q_at_draft = q_at_draft;
+    p.z_at_draft = stats + l.off_z; p.q_at_draft = stats + l.off_q;
     return launch_shard_gather_draft(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
-int massv_shard_scan(const massv_accept_desc* desc, int32_t world, int32_t n_partials_all, const float* part_max_all,
-                     const float* part_sum_all, const int32_t* part_idx_all, const int32_t* draft_tokens,
-                     const float* z_at_draft, const float* q_at_draft, const float* u_accept, int32_t* out_tokens,
-                     int32_t* accept_len, void* state, int32_t* dev_status, massv_stream_t stream) {
+int massv_shard_scan(const massv_accept_desc* desc, int32_t world, int32_t n_partials, const float* stats_all,
+                     const int32_t* draft_tokens, const float* u_accept, int32_t* out_tokens, int32_t* accept_len,
+                     void* state, int32_t* dev_status, massv_stream_t stream) {
     const int rc = check_shard(desc, world, 0);
     if (rc != MASSV_OK) return rc;
     const bool sampling = desc->temperature > 0.f;
-    if (n_partials_all < 1 || !part_max_all || !part_sum_all || !part_idx_all || !out_tokens || !accept_len || !state)
+    const ShardLayoutA l = shard_layout_a(*desc);
+    if (n_partials < 1 || n_partials > l.slots || !stats_all || !out_tokens || !accept_len || !state)
         return MASSV_ERR_INVALID_ARG;
-    if (desc->gamma > 0 && (!draft_tokens || (sampling && (!z_at_draft || !q_at_draft || !u_accept))))
-        return MASSV_ERR_INVALID_ARG;
+    if (desc->gamma > 0 && (!draft_tokens || (sampling && !u_accept))) return MASSV_ERR_INVALID_ARG;
     AcceptParams a{};
     a.B = desc->batch; a.gamma = desc->gamma; a.V = world * desc->vocab; a.T = desc->temperature;
-    a.n_part = n_partials_all;
-    a.part_max = const_cast<float*>(part_max_all); a.part_sum = const_cast<float*>(part_sum_all);
-    a.part_idx = const_cast<int32_t*>(part_idx_all);
+    a.n_part = world * n_partials; a.part_per_rank = n_partials; a.ranks = world; a.rank_stride = l.words;
+    a.part_max = const_cast<float*>(stats_all + l.off_max); a.part_sum = const_cast<float*>(stats_all + l.off_sum);
+    a.part_idx = reinterpret_cast<int32_t*>(const_cast<float*>(stats_all + l.off_idx));
     a.draft_tokens = draft_tokens; a.u_accept = u_accept;
-    a.z_at_draft = sampling ? z_at_draft : nullptr; a.q_at_draft = sampling ? q_at_draft : nullptr;
+    if (sampling) { a.z_at_draft = stats_all + l.off_z; a.q_at_draft = stats_all + l.off_q; }
     a.out_tokens = out_tokens; a.accept_len = accept_len;
     a.seq_state = static_cast<SeqState*>(state);
     a.dev_status = dev_status;
@@ -310,42 +336,40 @@ int massv_shard_scan(const massv_accept_desc* desc, int32_t world, int32_t n_par
 }
 
 int massv_shard_masses(const massv_accept_desc* desc, int32_t world, int32_t rank, const float* logits_shard,
-                       const float* draft_probs_shard, const void* state, double* mass_residual, double* mass_p,
-                       int32_t* dev_status, massv_stream_t stream) {
+                       const float* draft_probs_shard, const void* state, double* masses, int32_t* dev_status,
+                       massv_stream_t stream) {
     const int rc = check_shard(desc, world, rank);
     if (rc != MASSV_OK) return rc;
     if (!(desc->temperature > 0.f)) return MASSV_ERR_INVALID_ARG;
-    if (!logits_shard || !state || !mass_residual || !mass_p || (desc->gamma > 0 && !draft_probs_shard))
-        return MASSV_ERR_INVALID_ARG;
+    if (!logits_shard || !state || !masses || (desc->gamma > 0 && !draft_probs_shard)) return MASSV_ERR_INVALID_ARG;
     ShardParams p = shard_params(desc, world, rank, dev_status);
     p.logits = logits_shard; p.draft_probs = draft_probs_shard; p.seq_state = static_cast<const SeqState*>(state);
-    p.sums_res = mass_residual; p.sums_p = mass_p;
+    p.sums_res = masses; p.sums_p = masses + (size_t)desc->batch * p.n_chunks;
     return launch_shard_masses(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
-int massv_shard_pick(const massv_accept_desc* desc, int32_t world, int32_t rank, const double* mass_residual_all,
-                     const double* mass_p_all, const float* u_sample, const void* state, const float* logits_shard,
+int massv_shard_pick(const massv_accept_desc* desc, int32_t world, int32_t rank, const double* masses_all,
+                     const float* u_sample, const void* state, const float* logits_shard,
                      const float* draft_probs_shard, int32_t* token_out, int32_t* dev_status, massv_stream_t stream) {
     const int rc = check_shard(desc, world, rank);
     if (rc != MASSV_OK) return rc;
     if (!(desc->temperature > 0.f)) return MASSV_ERR_INVALID_ARG;
-    if (!mass_residual_all || !mass_p_all || !u_sample || !state || !logits_shard || !token_out ||
-        (desc->gamma > 0 && !draft_probs_shard))
+    if (!masses_all || !u_sample || !state || !logits_shard || !token_out || (desc->gamma > 0 && !draft_probs_shard))
         return MASSV_ERR_INVALID_ARG;
     ShardParams p = shard_params(desc, world, rank, dev_status);
-    if ((long)world * p.n_chunks > 512) return MASSV_ERR_UNSUPPORTED;
     p.logits = logits_shard; p.draft_probs = draft_probs_shard; p.seq_state = static_cast<const SeqState*>(state);
-    p.all_res = mass_residual_all; p.all_p = mass_p_all; p.u_sample = u_sample; p.token_out = token_out;
+    p.all_res = masses_all; p.all_p = masses_all + (size_t)desc->batch * p.n_chunks;
+    p.u_sample = u_sample; p.token_out = token_out;
     return launch_shard_pick(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
-int massv_shard_set_token(const massv_accept_desc* desc, const void* state, const int32_t* tokens, int32_t* out_tokens,
-                          int32_t* dev_status, massv_stream_t stream) {
-    const int rc = check_accept_desc(desc);
+int massv_shard_set_token(const massv_accept_desc* desc, int32_t world, const void* state, const int32_t* tokens_all,
+                          int32_t* out_tokens, int32_t* dev_status, massv_stream_t stream) {
+    const int rc = check_shard(desc, world, 0);
     if (rc != MASSV_OK) return rc;
-    if (!state || !tokens || !out_tokens) return MASSV_ERR_INVALID_ARG;
-    ShardParams p = shard_params(desc, 1, 0, dev_status);
-    p.seq_state = static_cast<const SeqState*>(state); p.tokens_in = tokens; p.out_tokens = out_tokens;
+    if (!state || !tokens_all || !out_tokens) return MASSV_ERR_INVALID_ARG;
+    ShardParams p = shard_params(desc, world, 0, dev_status);
+    p.seq_state = static_cast<const SeqState*>(state); p.tokens_in = tokens_all; p.out_tokens = out_tokens;
     return launch_shard_set_token(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 

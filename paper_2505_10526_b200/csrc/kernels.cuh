@@ -82,6 +82,11 @@ struct AcceptParams {
     // collected from the rank that owns the token (then `logits` / `draft_probs` are not read by the scan)
     const float* z_at_draft = nullptr;   // [B, gamma]
     const float* q_at_draft = nullptr;   // [B, gamma]
+    // gathered exchange buffers: partial slot i lives in rank i / part_per_rank's copy, the copies
+    // rank_stride words apart; z / q at the drafted tokens are the maximum over the ranks' copies
+    int part_per_rank = 0;               // 0: one contiguous [n_part, M] array
+    int ranks = 1;
+    size_t rank_stride = 0;              // in 4-byte words
 };
 cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream);
 cudaError_t launch_accept_scan_only(const AcceptParams& p, cudaStream_t stream);
@@ -99,12 +104,13 @@ struct ShardParams {
     double *sums_res, *sums_p;      // [B, n_chunks]: chunk masses of max(p - q, 0) and of p on the sampled row
     int n_chunks;                   // chunks of this shard
     // pick
-    const double *all_res, *all_p;  // [world, B, n_chunks]: ranks in order are vocabulary order
+    const double *all_res, *all_p;  // rank r's [B, n_chunks] at + r * mass_rank_stride: ranks in order are vocabulary order
+    size_t mass_rank_stride;        // in doubles
     int world, rank;
     const float* u_sample;          // [B, gamma+1]
     int32_t* token_out;             // [B]: the drawn token if this shard owns it, else -1
     int32_t* out_tokens;            // [B, gamma+1]
-    const int32_t* tokens_in;       // [B]
+    const int32_t* tokens_in;       // [world, B]: -1 from the ranks that do not own the token
     int32_t* dev_status;
 };
 cudaError_t launch_shard_gather_draft(const ShardParams& p, cudaStream_t stream);

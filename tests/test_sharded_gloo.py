@@ -1,6 +1,6 @@
 """The exchange of the vocabulary-sharded acceptance on two CPU ranks (gloo): the communicator's gather is
-rank-major, its reduction is a maximum, and a rank's phase generator is driven to the end with every rank
-seeing the same gathered values.  No kernel runs here; the phases are a stand-in that only exchanges."""
+rank-major and a rank's phase generator is driven to the end with every rank seeing the same gathered
+values.  No kernel runs here; the phases are a stand-in that only exchanges."""
 import os
 
 import torch
@@ -9,9 +9,9 @@ import torch.multiprocessing as mp
 
 
 def _phases(rank):
-    a = yield ("gather", torch.full((2, 3), float(rank)))
-    b = yield ("max", torch.tensor([rank * 10, -1 if rank == 0 else 7], dtype=torch.int32))
-    c = yield ("gather", torch.arange(4, dtype=torch.float64).view(1, 2, 2) + 100 * rank)
+    a = yield torch.full((6,), float(rank))
+    b = yield torch.tensor([rank * 10, -1 if rank == 0 else 7], dtype=torch.int32)
+    c = yield torch.arange(4, dtype=torch.float64) + 100 * rank
     return a, b, c
 
 
@@ -37,9 +37,9 @@ def test_two_ranks_exchange_in_rank_order():
         res = dict(out)
     assert res[0] == res[1]                                       # every rank sees the same values
     a, b, c = res[0]
-    assert a == [[0.0] * 3] * 2 + [[1.0] * 3] * 2                 # rank 0's rows, then rank 1's
-    assert b == [10, 7]
-    assert c == [[[0.0, 1.0], [2.0, 3.0]], [[100.0, 101.0], [102.0, 103.0]]]
+    assert a == [0.0] * 6 + [1.0] * 6                             # rank 0's copy, then rank 1's
+    assert b == [0, -1, 10, 7]
+    assert c == [0.0, 1.0, 2.0, 3.0, 100.0, 101.0, 102.0, 103.0]
 
 
 def test_lockstep_driver_matches_the_collectives():
@@ -57,6 +57,6 @@ def test_lockstep_driver_matches_the_collectives():
 
     res = run_lockstep([Rank(0), Rank(1)], [{}, {}])
     for a, b, c in res:
-        assert a.tolist() == [[0.0] * 3] * 2 + [[1.0] * 3] * 2
-        assert b.tolist() == [10, 7]
-        assert c.shape == (2, 2, 2) and c[1, 0, 0] == 100.0
+        assert a.tolist() == [0.0] * 6 + [1.0] * 6
+        assert b.tolist() == [0, -1, 10, 7]
+        assert c.tolist() == [0.0, 1.0, 2.0, 3.0, 100.0, 101.0, 102.0, 103.0]
