@@ -322,6 +322,20 @@ int massv_shard_set_token(const massv_accept_desc *desc, int32_t world, const vo
                           const int32_t *tokens_all, int32_t *out_tokens, int32_t *dev_status,
                           massv_stream_t stream);
 
+/*
+ * The all-gather of the sharded acceptance done by this library's own kernel instead of a collective
+ * library: one launch stores `bytes` bytes of src at offset rank * bytes of each of the `world`
+ * gathered buffers.  gathered is a HOST array of world device pointers; entry w is rank w's gathered
+ * buffer as seen from this GPU (its own for w == rank, peer-mapped memory for the others: a symmetric
+ * allocation or an IPC mapping), each world * bytes long.  Plain stores only.  The call orders nothing
+ * between ranks: a rank may read its gathered buffer only after every rank's publish has completed
+ * (the caller's barrier), and may publish into it again only after every rank has finished reading.
+ * bytes % 4 == 0; pointers 4-byte aligned (16-byte aligned buffers and sizes copy 16 bytes per store);
+ * world <= 16.
+ */
+int massv_shard_publish(const void *src, size_t bytes, void *const *gathered, int32_t world, int32_t rank,
+                        massv_stream_t stream);
+
 /* Human-readable name of a massv_status value. */
 const char *massv_strerror(int status);
 

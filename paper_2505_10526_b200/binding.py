@@ -74,6 +74,8 @@ def _load():
     lib.massv_shard_masses.argtypes = [D, i32, i32, f32p, f32p, vp, vp, i32p, vp]
     lib.massv_shard_pick.restype = ctypes.c_int
     lib.massv_shard_pick.argtypes = [D, i32, i32, vp, f32p, vp, f32p, f32p, i32p, i32p, vp]
+    lib.massv_shard_publish.restype = ctypes.c_int
+    lib.massv_shard_publish.argtypes = [vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_void_p), i32, i32, vp]
     lib.massv_shard_set_token.restype = ctypes.c_int
     lib.massv_shard_set_token.argtypes = [D, i32, vp, i32p, i32p, i32p, vp]
     lib.massv_kv_commit.restype = ctypes.c_int
@@ -282,6 +284,17 @@ def massv_shard_pick(desc, world, rank, masses_all, u_sample, state, logits_shar
     _check(_lib.massv_shard_pick(ctypes.byref(desc), world, rank, _ptr(masses_all, f64), _ptr(u_sample, f32),
                                  _ptr(state, torch.uint8), _ptr(logits_shard, f32), _ptr(draft_probs_shard, f32),
                                  _ptr(token_out, i32), _ptr(dev_status, i32), _stream()), "massv_shard_pick")
+
+
+def massv_shard_publish(src, gathered, rank) -> None:
+    """Store ``src`` at slot ``rank`` of every tensor in ``gathered`` (one per rank, each world x src's size)."""
+    world = len(gathered)
+    nbytes = src.numel() * src.element_size()
+    for g in gathered:
+        if g.numel() * g.element_size() != world * nbytes:
+            raise ValueError("massv: a gathered buffer must be world times the source's size")
+    ptrs = (ctypes.c_void_p * world)(*[_ptr(g) for g in gathered])
+    _check(_lib.massv_shard_publish(_ptr(src), nbytes, ptrs, world, rank, _stream()), "massv_shard_publish")
 
 
 def massv_shard_set_token(desc, world, state, tokens_all, out_tokens, dev_status=None) -> None:

@@ -456,6 +456,23 @@ __global__ void shard_set_token_kernel(ShardParams p) {
     p.out_tokens[(size_t)b * (p.gamma + 1) + p.seq_state[b].n] = tok;
 }
 
+// grid (blocks, world): block column w copies this rank's buffer into rank w's gathered buffer.  Plain
+// stores: the destination may be another GPU's memory mapped into this one's address space.
+__global__ void shard_publish_kernel(PublishParams p) {
+    pdl_wait();
+    char* dst = static_cast<char*>(p.dst[blockIdx.y]) + (size_t)p.rank * p.bytes;
+    const char* src = static_cast<const char*>(p.src);
+    const size_t stride = (size_t)gridDim.x * blockDim.x, first = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool wide = p.bytes % 16 == 0 && (reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(p.dst[blockIdx.y])) % 16 == 0;
+    if (wide) {
+        for (size_t i = first; i < p.bytes / 16; i += stride)
+            reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
+    } else {
+        for (size_t i = first; i < p.bytes / 4; i += stride)
+            reinterpret_cast<uint32_t*>(dst)[i] = reinterpret_cast<const uint32_t*>(src)[i];
+    }
+}
+
 // Dense probabilities for callers that ask for them (diagnostics / tests).
 __global__ void probs_kernel(AcceptParams p) {
     const int R = p.gamma + 1, M = p.B * R;
@@ -534,6 +551,16 @@ cudaError_t launch_shard_pick(const ShardParams& p, cudaStream_t stream) {
 }
 cudaError_t launch_shard_set_token(const ShardParams& p, cudaStream_t stream) {
     if (launch_pdl(shard_set_token_kernel, dim3((p.B + 127) / 128), dim3(128), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_shard_publish(const PublishParams& p, cudaStream_t stream) {
+    if (p.bytes == 0) return cudaSuccess;
+    size_t blocks = (p.bytes / 16 + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 64) blocks = 64;
+    if (launch_pdl(shard_publish_kernel, dim3((unsigned)blocks, p.world), dim3(256), 0, stream, p) != cudaSuccess) return cudaGetLastError();
     count_launches(1);
     return cudaGetLastError();
 }

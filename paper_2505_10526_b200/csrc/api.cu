@@ -373,6 +373,19 @@ int massv_shard_set_token(const massv_accept_desc* desc, int32_t world, const vo
     return launch_shard_set_token(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
+int massv_shard_publish(const void* src, size_t bytes, void* const* gathered, int32_t world, int32_t rank,
+                        massv_stream_t stream) {
+    if (world < 1 || world > kMaxPeers || rank < 0 || rank >= world) return world > kMaxPeers ? MASSV_ERR_UNSUPPORTED : MASSV_ERR_INVALID_ARG;
+    if (!src || !gathered || bytes % 4 != 0 || reinterpret_cast<uintptr_t>(src) % 4 != 0) return MASSV_ERR_INVALID_ARG;
+    PublishParams p{};
+    p.src = src; p.bytes = bytes; p.world = world; p.rank = rank;
+    for (int w = 0; w < world; ++w) {
+        if (!gathered[w] || reinterpret_cast<uintptr_t>(gathered[w]) % 4 != 0) return MASSV_ERR_INVALID_ARG;
+        p.dst[w] = gathered[w];
+    }
+    return launch_shard_publish(p, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
 size_t massv_tvd_workspace_size(const massv_accept_desc* desc) {
     if (check_accept_desc(desc) != MASSV_OK || desc->gamma < 1 || !(desc->temperature > 0.f)) return 0;
     const size_t rows = (size_t)desc->batch * desc->gamma;

@@ -118,6 +118,16 @@ cudaError_t launch_shard_masses(const ShardParams& p, cudaStream_t stream);
 cudaError_t launch_shard_pick(const ShardParams& p, cudaStream_t stream);
 cudaError_t launch_shard_set_token(const ShardParams& p, cudaStream_t stream);
 
+// An all-gather by stores: this rank's buffer goes to offset rank * bytes of every rank's gathered buffer.
+constexpr int kMaxPeers = 16;
+struct PublishParams {
+    const void* src;
+    size_t bytes;                   // multiple of 4
+    void* dst[kMaxPeers];           // the ranks' gathered buffers (peer-mapped device pointers)
+    int world, rank;
+};
+cudaError_t launch_shard_publish(const PublishParams& p, cudaStream_t stream);
+
 // ---------------------------------------------------------------- TVD diagnostic
 constexpr int kTvdSlices = 16;      // vocabulary slices per row
 struct TvdParams {

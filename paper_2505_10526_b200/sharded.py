@@ -6,7 +6,9 @@ three small exchange buffers between ranks (three all-gathers per step, one at t
 
 * ``DistComm``  -- ``torch.distributed`` collectives (NCCL between GPUs; gloo in the CPU tests);
 * ``run_lockstep`` -- all ranks of a world on ONE device, phase by phase, concatenation in place of the
-  all-gather: the single-GPU check of the multi-rank path (no rank's kernel waits on another's).
+  all-gather: the single-GPU check of the multi-rank path (no rank's kernel waits on another's).  Its
+  "publish" transport uses the library's own all-gather-by-stores kernel (``massv_shard_publish``), the
+  ranks' gathered buffers standing for peer-mapped memory.
 
 The phases are a generator's steps: a rank yields the buffer it wants gathered and is resumed with the
 gathered one, so both transports drive the same code.
@@ -44,17 +46,27 @@ def drive(phases, comm):
         return e.value
 
 
-def run_lockstep(ranks, inputs):
-    """All ranks on one device: advance every rank to its next exchange, concatenate, resume.
-    ``ranks``: list of ShardedAccept in rank order; ``inputs``: per-rank kwargs of ``phases``."""
+def run_lockstep(ranks, inputs, transport="concat"):
+    """All ranks on one device: advance every rank to its next exchange, combine, resume.
+    ``ranks``: list of ShardedAccept in rank order; ``inputs``: per-rank kwargs of ``phases``.
+    ``transport``: "concat" (concatenation stands for the collective) or "publish" (every rank stores its
+    buffer into every rank's gathered buffer with ``massv_shard_publish``; stream order on the one device
+    stands for the barrier between publishing and reading)."""
     gens = [r.phases(**kw) for r, kw in zip(ranks, inputs)]
     reqs = [next(g) for g in gens]
     while True:
-        gathered = torch.cat(reqs, dim=0)
+        if transport == "publish":
+            world = len(reqs)
+            bufs = [torch.empty((world * t.numel(),), dtype=t.dtype, device=t.device) for t in reqs]
+            for r, t in enumerate(reqs):
+                mv.massv_shard_publish(t, bufs, r)
+        else:
+            cat = torch.cat(reqs, dim=0)
+            bufs = [cat.clone() for _ in reqs]
         nxt, done = [], []
-        for g in gens:
+        for g, buf in zip(gens, bufs):
             try:
-                nxt.append(g.send(gathered.clone()))
+                nxt.append(g.send(buf))
             except StopIteration as e:
                 done.append(e.value)
         if done:

@@ -18,7 +18,7 @@ from workloads import generate, get_config
 pytestmark = pytest.mark.gpu
 
 
-def _run_sharded(cfg, w, world):
+def _run_sharded(cfg, w, world, transport="concat"):
     from paper_2505_10526_b200.sharded import ShardedAccept, run_lockstep
     assert cfg.vocab % world == 0
     Vs = cfg.vocab // world
@@ -31,7 +31,7 @@ def _run_sharded(cfg, w, world):
             kw.update(draft_probs_shard=w["draft_probs"][:, :, r * Vs:(r + 1) * Vs].contiguous(),
                       u_accept=w["u_accept"], u_sample=w["u_sample"])
         inputs.append(kw)
-    res = run_lockstep(ranks, inputs)
+    res = run_lockstep(ranks, inputs, transport=transport)
     torch.cuda.synchronize()
     for rk in ranks:
         assert int(rk.dev_status.item()) == 0
@@ -41,9 +41,9 @@ def _run_sharded(cfg, w, world):
     return toks, lens, ranks
 
 
-def _check(cfg, world, subset=None, w=None):
+def _check(cfg, world, subset=None, w=None, transport="concat"):
     w = w or generate(cfg, device="cuda", with_attention=False)
-    toks, lens, ranks = _run_sharded(cfg, w, world)
+    toks, lens, ranks = _run_sharded(cfg, w, world, transport)
     idx = list(range(cfg.batch)) if subset is None else subset
     ref = oracle.verify_step(sub_workload(w, idx), cfg.temperature, want_attention=False)
     sel = torch.as_tensor(idx, device="cuda")
@@ -92,6 +92,31 @@ def test_every_draft_accepted_draws_the_bonus_token_across_shards():
     w["u_accept"].zero_()
     toks, lens = _check(cfg, 2, w=w)
     assert bool((lens == cfg.gamma + 1).all())
+
+
+@pytest.mark.parametrize("world", [1, 3, 8])
+@pytest.mark.parametrize("name", ["tiny_ragged_t0", "tiny_ragged_t1"])
+def test_own_all_gather_kernel_in_place_of_the_collective(name, world):
+    """The three exchanges done by massv_shard_publish (stores into every rank's gathered buffer).
+    tiny_ragged_t1 has batch 7: its token exchange is 28 bytes, the 4-byte store path."""
+    cfg = get_config(name)
+    cfg = replace(cfg, vocab=1024 * 3) if world == 3 else cfg
+    _check(cfg, world, transport="publish")
+
+
+def test_publish_places_every_rank_at_its_offset():
+    from paper_2505_10526_b200 import binding as mv
+    world, n = 4, 1000
+    src = [torch.arange(n, dtype=torch.int32, device="cuda") + 10000 * r for r in range(world)]
+    bufs = [torch.full((world * n,), -1, dtype=torch.int32, device="cuda") for _ in range(world)]
+    for r in range(world):
+        mv.massv_shard_publish(src[r], bufs, r)
+    torch.cuda.synchronize()
+    want = torch.cat(src)
+    for b in bufs:
+        assert torch.equal(b, want)
+    with pytest.raises(ValueError):
+        mv.massv_shard_publish(src[0], [bufs[0][:-4]] * world, 0)
 
 
 @pytest.mark.parametrize("name,world,subset", [("qwen7b_b1_t0", 2, None), ("qwen7b_b16_t1", 4, [0, 7, 15]),
