@@ -123,6 +123,17 @@ def tvd(p, q):
     return float(_load().oracle_tvd(p.shape[0], _p(p, np.float64), _p(q, np.float64)))
 
 
+def tvd_histogram(tvd, bins, counts=None):
+    """counts[k] += number of TVD values (f32, any shape) in bin k of `bins` equal bins over [0, 1]."""
+    t = np.ascontiguousarray(tvd, dtype=np.float32).reshape(-1)
+    if counts is None:
+        counts = np.zeros((bins,), dtype=np.int64)
+    lib = _load()
+    lib.oracle_tvd_histogram.restype = ctypes.c_longlong
+    lib.oracle_tvd_histogram(ctypes.c_longlong(t.shape[0]), _p(t, np.float32), int(bins), _p(counts, np.int64))
+    return counts
+
+
 def sample_top_p(z, u, T, top_p, want_q=True):
     """Nucleus sampling of softmax(z / T), row by row: z f32 [rows, V], u f32 [rows].
     Returns dict(token, q (f64 [rows, V] or None), nucleus_size, margin_set, margin_sample)."""

@@ -297,6 +297,28 @@ double oracle_tvd(int V, const double *p, const double *q)
 }
 
 /*
+ * Histogram of total variation distances (Fig. 4 plots the TVDs of Eq. 6 as a histogram): counts[k] +=
+ * the number of values in bin k of `bins` equal-width bins over [0, 1] -- bin k is [k / bins, (k+1) / bins),
+ * the last bin also takes 1.  The paper fixes neither the bin count nor the edges' arithmetic: the bin
+ * index is floor(t * bins) with the product rounded once to single precision (the type the distances
+ * are stored in), clamped to [0, bins - 1]; NaN values are not counted.  Returns the number counted.
+ */
+long long oracle_tvd_histogram(long long n, const float *tvd, int bins, long long *counts)
+{
+    long long counted = 0;
+    for (long long i = 0; i < n; ++i) {
+        const float t = tvd[i];
+        if (t != t) continue;
+        const float scaled = t * (float)bins;
+        int k = scaled <= 0.0f ? 0 : (scaled >= (float)bins ? bins - 1 : (int)scaled);
+        if (k > bins - 1) k = bins - 1;
+        counts[k] += 1;
+        ++counted;
+    }
+    return counted;
+}
+
+/*
  * Nucleus (top-p) sampling of softmax(z / T) (Sec. 3.2: the target's responses for self-distillation are
  * drawn as sample_top-p(p(. | I, X)); the same rule is the drafter's sampling step when it uses top-p).
  * Per row: order the tokens by probability, largest first (equal probabilities: lower index first); the

@@ -578,6 +578,29 @@ def test_tvd_hand_values():
     assert abs(oracle.tvd(a, b) - oracle.tvd(b, a)) < 1e-18
 
 
+def test_tvd_histogram_hand_values_and_library_histogram():
+    """Fig. 4's histogram of Eq. 6 values: hand-placed values, the closed right edge, accumulation over
+    calls, NaN skipped, and agreement with numpy's histogram on values away from the bin edges."""
+    vals = np.array([0.0, 0.049, 0.05, 0.5, 0.99, 1.0, 0.31, 0.31, np.nan], dtype=np.float32)
+    c = oracle.tvd_histogram(vals, 10)
+    assert c.tolist() == [3, 0, 0, 2, 0, 1, 0, 0, 0, 2]          # 0, .049, .05 | .31 x2 | .5 | .99 and 1.0
+    assert c.sum() == 8                                          # the NaN is not counted
+    c2 = oracle.tvd_histogram(np.array([0.05, 0.95], np.float32), 10, counts=c.copy())
+    assert c2.tolist() == [4, 0, 0, 2, 0, 1, 0, 0, 0, 3]         # accumulates
+    assert oracle.tvd_histogram(np.array([-1e-7, 1.0000001], np.float32), 4).tolist() == [1, 0, 0, 1]   # rounding strays
+    rng = np.random.default_rng(3)
+    for bins in (7, 20, 64):
+        # mid-points of a fine grid: at least 1/(2*4096*bins) away from every edge, far beyond fp32 rounding
+        k = rng.integers(0, 4096 * bins, size=5000)
+        v = ((k + 0.5) / (4096 * bins)).astype(np.float32)
+        want, _ = np.histogram(v.astype(np.float64), bins=bins, range=(0.0, 1.0))
+        assert np.array_equal(oracle.tvd_histogram(v, bins), want)
+    # a skewed sample keeps its shape: every TVD of identical distributions lands in bin 0
+    p = rng.dirichlet(np.ones(32), size=50)
+    t = np.array([oracle.tvd(p[i], p[i].copy()) for i in range(50)], np.float32)
+    assert oracle.tvd_histogram(t, 16)[0] == 50
+
+
 # ---------------------------------------------------------------- nucleus (top-p) sampling (Sec. 3.2)
 def _softmax64(z, T):
     z = z.astype(np.float64) / T
