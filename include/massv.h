@@ -242,6 +242,17 @@ int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t *accept_len, int
                     int32_t *dev_status, massv_stream_t stream);
 
 /*
+ * Histogram of TVD values, the form in which the paper presents Eq. 6 (Fig. 4): counts[k] += the number
+ * of tvd[i] in bin k of `bins` equal-width bins over [0, 1]; bin k is [k / bins, (k + 1) / bins), the last
+ * bin also takes 1.  The bin index is floor(tvd * bins) with the product rounded once in fp32, clamped to
+ * [0, bins - 1]; NaN is not counted.  counts is ADDED to (int64 [bins], device memory, zeroed by the
+ * caller before the first call), so one array can collect the tvd_out of many massv_tvd calls.
+ *   0 <= n <= 2^40;  1 <= bins <= 4096;  tvd fp32 [n] (for instance tvd_out of massv_tvd)
+ * No workspace.
+ */
+int massv_tvd_histogram(int64_t n, const float *tvd, int32_t bins, int64_t *counts, massv_stream_t stream);
+
+/*
  * Nucleus (top-p) sampling of softmax(z / T), row by row (Sec. 3.2: the target's responses for the
  * drafter's self-distillation are drawn as sample_top-p(p(. | I, X)); the same call is the drafter's
  * sampling step when it samples with top-p, probs_out then being the draft distribution q that

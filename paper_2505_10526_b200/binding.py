@@ -58,6 +58,8 @@ def _load():
     lib.massv_tvd_workspace_size.argtypes = [ctypes.POINTER(AcceptDesc)]
     lib.massv_tvd.restype = ctypes.c_int
     lib.massv_tvd.argtypes = [ctypes.POINTER(AcceptDesc), f32p, f32p, f32p, f32p, vp, ctypes.c_size_t, i32p, vp]
+    lib.massv_tvd_histogram.restype = ctypes.c_int
+    lib.massv_tvd_histogram.argtypes = [ctypes.c_int64, f32p, ctypes.c_int32, vp, vp]
     lib.massv_sample_top_p.restype = ctypes.c_int
     lib.massv_sample_top_p.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_float, f32p, f32p, i32p, f32p, i32p, vp]
     D, i32 = ctypes.POINTER(AcceptDesc), ctypes.c_int32
@@ -215,6 +217,13 @@ def massv_tvd(desc, logits, draft_probs, tvd_out, accept_prob_out=None, workspac
                         _ptr(dev_status, torch.int32), _stream())
     if rc != 0:
         raise MassvError(rc, "massv_tvd")
+
+
+def massv_tvd_histogram(tvd, counts) -> None:
+    """counts (int64 [bins]) += histogram of the fp32 tensor ``tvd`` over [0, 1]."""
+    rc = _lib.massv_tvd_histogram(tvd.numel(), _ptr(tvd, torch.float32), counts.numel(), _ptr(counts, torch.int64), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_tvd_histogram")
 
 
 def massv_sample_top_p(logits, u, tokens, temperature, top_p, probs_out=None, dev_status=None) -> None:

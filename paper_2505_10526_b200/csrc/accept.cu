@@ -456,6 +456,28 @@ __global__ void shard_set_token_kernel(ShardParams p) {
     p.out_tokens[(size_t)b * (p.gamma + 1) + p.seq_state[b].n] = tok;
 }
 
+// Histogram of TVD values: per-CTA counts in shared memory, one global atomic per non-empty bin and CTA.
+constexpr int kHistMaxBins = 4096;
+__global__ void __launch_bounds__(256) tvd_histogram_kernel(long long n, const float* __restrict__ tvd, int bins,
+                                                            unsigned long long* counts) {
+    extern __shared__ unsigned int s_hist[];
+    for (int k = threadIdx.x; k < bins; k += blockDim.x) s_hist[k] = 0u;
+    pdl_wait();
+    __syncthreads();
+    const float fb = (float)bins;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const float t = tvd[i];
+        if (t != t) continue;
+        const float scaled = __fmul_rn(t, fb);               // one rounding, never contracted
+        int k = scaled <= 0.f ? 0 : (scaled >= fb ? bins - 1 : (int)scaled);
+        k = min(k, bins - 1);
+        atomicAdd(&s_hist[k], 1u);
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < bins; k += blockDim.x)
+        if (s_hist[k]) atomicAdd(&counts[k], (unsigned long long)s_hist[k]);
+}
+
 // grid (blocks, world): block column w copies this rank's buffer into rank w's gathered buffer.  Plain
 // stores: the destination may be another GPU's memory mapped into this one's address space.
 __global__ void shard_publish_kernel(PublishParams p) {
@@ -551,6 +573,19 @@ cudaError_t launch_shard_pick(const ShardParams& p, cudaStream_t stream) {
 }
 cudaError_t launch_shard_set_token(const ShardParams& p, cudaStream_t stream) {
     if (launch_pdl(shard_set_token_kernel, dim3((p.B + 127) / 128), dim3(128), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_tvd_histogram(long long n, const float* tvd, int bins, unsigned long long* counts, cudaStream_t stream) {
+    if (n == 0) return cudaSuccess;
+    if (bins > kHistMaxBins) return cudaErrorInvalidValue;
+    long long blocks = (n + 255) / 256;
+    if (blocks > 2 * 148) blocks = 2 * 148;
+    // a CTA sees fewer than 2^32 values: its shared counters are 32-bit
+    if (launch_pdl(tvd_histogram_kernel, dim3((unsigned)blocks), dim3(256), (size_t)bins * sizeof(unsigned int), stream, n, tvd, bins,
+                   counts) != cudaSuccess)
+        return cudaGetLastError();
     count_launches(1);
     return cudaGetLastError();
 }

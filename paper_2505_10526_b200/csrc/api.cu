@@ -415,6 +415,14 @@ int massv_tvd(const massv_accept_desc* desc, const float* logits, const float* d
     return launch_tvd(t, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
 }
 
+int massv_tvd_histogram(int64_t n, const float* tvd, int32_t bins, int64_t* counts, massv_stream_t stream) {
+    if (n < 0 || bins < 1 || !counts || (n > 0 && !tvd)) return MASSV_ERR_INVALID_ARG;
+    if (bins > 4096 || n > ((int64_t)1 << 40)) return MASSV_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(counts) % 8 != 0) return MASSV_ERR_INVALID_ARG;
+    return launch_tvd_histogram((long long)n, tvd, bins, reinterpret_cast<unsigned long long*>(counts),
+                                reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
 int massv_sample_top_p(int32_t rows, int32_t vocab, float temperature, float top_p, const float* logits, const float* u,
                        int32_t* tokens, float* probs_out, int32_t* dev_status, massv_stream_t stream) {
     if (rows < 1 || vocab < 1 || !(temperature > 0.f) || !(top_p > 0.f) || !(top_p <= 1.f)) return MASSV_ERR_INVALID_ARG;

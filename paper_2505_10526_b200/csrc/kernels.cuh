@@ -118,6 +118,9 @@ cudaError_t launch_shard_masses(const ShardParams& p, cudaStream_t stream);
 cudaError_t launch_shard_pick(const ShardParams& p, cudaStream_t stream);
 cudaError_t launch_shard_set_token(const ShardParams& p, cudaStream_t stream);
 
+// counts[k] += number of tvd values in bin k of `bins` equal bins over [0, 1] (NaN not counted)
+cudaError_t launch_tvd_histogram(long long n, const float* tvd, int bins, unsigned long long* counts, cudaStream_t stream);
+
 // An all-gather by stores: this rank's buffer goes to offset rank * bytes of every rank's gathered buffer.
 constexpr int kMaxPeers = 16;
 struct PublishParams {

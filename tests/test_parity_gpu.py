@@ -329,6 +329,58 @@ def test_tvd_diagnostic_matches_oracle(name, subset):
             assert 0.0 <= float(tvd[b, j]) <= 1.0 + 1e-6
 
 
+@pytest.mark.parametrize("n,bins", [(0, 8), (1, 1), (1000, 10), (100003, 50), (3_000_000, 4096), (70001, 37)])
+def test_tvd_histogram_matches_oracle(n, bins):
+    """Bit-exact counts: both sides take the bin from one fp32 product.  Values are a skewed mix on [0, 1]
+    with exact edges (0, 1, k / bins), strays just outside, and NaN; a second call accumulates."""
+    import paper_2505_10526_b200 as mv
+    gen = torch.Generator(device="cpu"); gen.manual_seed(1000 + n + bins)
+    v = torch.rand((n,), generator=gen, dtype=torch.float32) ** 3            # concentrated at low values, as in Fig. 4
+    if n >= 1000:
+        v[:bins] = torch.arange(bins, dtype=torch.float32) / bins             # exact edges
+        v[bins] = 1.0; v[bins + 1] = 0.0; v[bins + 2] = float("nan"); v[bins + 3] = 1.0000001; v[bins + 4] = -1e-8
+    dv = v.cuda()
+    counts = torch.zeros((bins,), dtype=torch.int64, device="cuda")
+    mv.massv_tvd_histogram(dv, counts)
+    torch.cuda.synchronize()
+    want = oracle.tvd_histogram(v.numpy(), bins)
+    assert np.array_equal(counts.cpu().numpy(), want)
+    assert int(counts.sum()) == n - (1 if n >= 1000 else 0)
+    mv.massv_tvd_histogram(dv, counts)
+    torch.cuda.synchronize()
+    assert np.array_equal(counts.cpu().numpy(), 2 * want)
+
+
+def test_tvd_histogram_of_a_verify_steps_distances():
+    """massv_tvd's output through massv_tvd_histogram equals the oracle's histogram of the same fp32 values,
+    and of the oracle's own distances wherever those are not within 1e-4 of a bin edge."""
+    import paper_2505_10526_b200 as mv
+    cfg = get_config("tiny_ragged_t1")
+    w = generate(cfg, device="cuda", with_attention=False)
+    B, R, g, V = cfg.batch, cfg.rows, cfg.gamma, cfg.vocab
+    desc = mv.accept_desc(B, g, cfg.hidden, V, cfg.temperature)
+    ws = mv.alloc_workspace(mv.massv_accept_workspace_size(desc), "cuda")
+    toks = torch.zeros((B, R), dtype=torch.int32, device="cuda"); lens = torch.zeros((B,), dtype=torch.int32, device="cuda")
+    logits = torch.zeros((B, R, V), dtype=torch.float32, device="cuda")
+    mv.massv_accept(desc, w["hidden"], w["lm_head"], w["draft_tokens"], w["draft_probs"], w["u_accept"], w["u_sample"],
+                    toks, lens, logits, None, ws, None)
+    tvd = torch.zeros((B, g), dtype=torch.float32, device="cuda")
+    mv.massv_tvd(desc, logits, w["draft_probs"], tvd, None, mv.alloc_workspace(mv.massv_tvd_workspace_size(desc), "cuda"), None)
+    bins = 8
+    counts = torch.zeros((bins,), dtype=torch.int64, device="cuda")
+    mv.massv_tvd_histogram(tvd, counts)
+    torch.cuda.synchronize()
+    assert np.array_equal(counts.cpu().numpy(), oracle.tvd_histogram(tvd.cpu().numpy(), bins))
+    p = oracle.softmax(oracle.logits(oracle.bf16_bits(w["hidden"]).reshape(B * R, cfg.hidden), oracle.bf16_bits(w["lm_head"])),
+                       cfg.temperature).reshape(B, R, V)
+    q = w["draft_probs"].double().cpu().numpy()
+    ref = np.array([[oracle.tvd(np.ascontiguousarray(p[b, j]), np.ascontiguousarray(q[b, j])) for j in range(g)] for b in range(B)])
+    clear = np.abs(ref * bins - np.round(ref * bins)) > 1e-4 * bins
+    got_bins = np.minimum((tvd.cpu().numpy() * np.float32(bins)).astype(np.int64), bins - 1)
+    assert np.array_equal(got_bins[clear], np.minimum((ref * bins).astype(np.int64), bins - 1)[clear])
+    assert int(counts.sum()) == B * g
+
+
 def test_gamma_zero_sampling_is_the_draft_side_step():
     """With no drafts and T > 0 the call is one ordinary sampling step: the token is the
     inverse-CDF draw from softmax(z / T) with the caller's uniform, and probs_out is that
