@@ -124,3 +124,21 @@ def test_publish_places_every_rank_at_its_offset():
 def test_full_size_vocabulary(name, world, subset):
     cfg = get_config(name)
     _check(cfg, world, subset=subset)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_small_shapes(seed):
+    """Seeded random geometry: 1 to 8 ranks, shard sizes off the 128-row tile and off the 4096-entry chunk,
+    gamma 0 to 7, greedy and sampled, flat and peaked target distributions, either transport."""
+    import random
+    from workloads import VerifyConfig
+    rnd = random.Random(9100 + seed)
+    world = rnd.choice([1, 2, 3, 4, 6, 8])
+    gamma = rnd.randint(0, 7)
+    batch = rnd.choice([1, 2, 3, 5, 9, 17])
+    shard = 8 * rnd.choice([16, 37, 100, 513, 1030])
+    cfg = VerifyConfig(name=f"shardfuzz{seed}", batch=batch, gamma=gamma, n_q_heads=4, n_kv_heads=1, head_dim=64,
+                       hidden=64 * rnd.randint(1, 6), vocab=shard * world, temperature=rnd.choice([0.0, 0.6, 1.0, 1.4]),
+                       ctx_lo=8, ctx_hi=8, image_tokens=0.25, draft_noise_std=rnd.choice([0.3, 1.0]), seed=9100 + seed,
+                       hidden_std=rnd.choice([1.0, 6.0]))
+    _check(cfg, world, transport=rnd.choice(["concat", "publish"]))
