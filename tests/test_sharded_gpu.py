@@ -142,3 +142,33 @@ def test_random_small_shapes(seed):
                        ctx_lo=8, ctx_hi=8, image_tokens=0.25, draft_noise_std=rnd.choice([0.3, 1.0]), seed=9100 + seed,
                        hidden_std=rnd.choice([1.0, 6.0]))
     _check(cfg, world, transport=rnd.choice(["concat", "publish"]))
+
+
+@pytest.mark.parametrize("world", [1, 2, 4])
+def test_empty_residual_falls_back_to_the_target_distribution(world):
+    """p = q = one-hot on token 700 (a logit gap of 1024 underflows every other probability to zero, in
+    fp32 and in fp64 alike), the drafted token is another one with p = q = 0: u * q < p fails, the draft is
+    rejected, and max(p - q, 0) has no mass on any shard.  Both sides must then draw from p: token 700,
+    whichever shard it lives on.  The unsharded call must agree too."""
+    from paper_2505_10526_b200 import VerifyStep
+    cfg = replace(get_config("tiny_t1"), batch=2, gamma=2, seed=3)
+    w = generate(cfg, device="cuda", with_attention=False)
+    V, K, hot = cfg.vocab, cfg.hidden, 700
+    w["hidden"].fill_(2.0)
+    w["lm_head"].zero_()
+    w["lm_head"][hot].fill_(2.0)                               # z[hot] = 4 K = 1024, every other logit 0
+    w["draft_probs"].zero_()
+    w["draft_probs"][:, :, hot] = 1.0
+    w["draft_tokens"].copy_(torch.tensor([[5, hot], [hot, 900]], dtype=torch.int32))
+    ref = oracle.verify_step(w, cfg.temperature, want_attention=False)
+    assert ref["accept_len"].tolist() == [1, 2]
+    assert ref["out_tokens"][0, 0] == hot and ref["out_tokens"][1].tolist()[:2] == [hot, hot]
+    toks, lens, _ = _run_sharded(cfg, w, world)
+    assert lens.tolist() == [1, 2]
+    assert int(toks[0, 0]) == hot and toks[1].tolist()[:2] == [hot, hot]
+    wa = dict(w)
+    wa.update(generate(cfg, device="cuda", with_lm_head=False))  # attention inputs for the whole-step object
+    step = VerifyStep.for_workload(cfg, wa)
+    step.run(wa, commit=False)
+    torch.cuda.synchronize()
+    assert torch.equal(step.accept_len, lens) and torch.equal(step.out_tokens, toks)
