@@ -33,6 +33,7 @@ constexpr int kTileBytesW = kVocabTile * kBlockK * 2;
 constexpr int kMaxStages = 12;
 constexpr int kMaxCtas = 192;               // partial slots are sized for at most this many CTAs
 constexpr int kRingBytes = 200 * 1024;      // shared memory given to the TMA ring
+constexpr int kPrefetchBlocks = 32;         // K blocks (16 KB each) of the first tile hinted into L2 before the dependency wait
 constexpr int kPairMinTile = 64;            // token rows per tile from which CTA pairs are used
 
 struct UmmaParams {
@@ -303,6 +304,16 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     volatile int* abort_ptr = &abort_flag;
+    // The weights do not depend on the kernel before this one: while it drains, an epilogue warp (idle
+    // until the first accumulator is ready) asks L2 for the first boxes of this CTA's first tile.
+    // Single-CTA tiles only: with CTA pairs the hints cost more than they bring.  Depth by measurement:
+    // the step gains up to 32 boxes (-2.4 %), beyond 40 the hinted boxes are fetched twice too often.
+    if constexpr (!PAIR) {
+        if (warp == 2 && lane == 0 && n_tiles > 0) {
+            const int n_pf = min(num_kb, kPrefetchBlocks);
+            for (int kb = 0; kb < n_pf; ++kb) tma_prefetch_2d(&map_w128, kb * kBlockK, row_begin);
+        }
+    }
     pdl_wait();          // everything above overlapped with the tail of the previous kernel
 
     if (warp == 0) {

@@ -56,6 +56,11 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
         : "memory");
 }
 
+// A hint to bring one box of a tensor map into L2; nothing waits on it and nothing in shared memory changes.
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
+
 // Host: 2-D bf16 tensor map over [rows, cols] (cols contiguous) with a box of
 // [box_rows, 64 cols] and the 128-byte swizzle.  Returns false if the driver
 // entry point is unavailable or rejects the shape.
