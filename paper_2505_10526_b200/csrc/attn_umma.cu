@@ -677,7 +677,8 @@ __global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(
     const int n = c_last - c_first + 1;
     auto slot_of = [&](int i) -> size_t { const int c = c_first + i; return (size_t)c * 2 + (start <= c * per_cta ? 0 : 1); };
     // per row: the common maximum and 1 / sum; per (piece, row): the merge weight
-    extern __shared__ float s_comb[];
+    extern __shared__ float4 s_red[];              // [kFlatCombineThreads]: partial sums of the piece groups (below)
+    float* s_comb = reinterpret_cast<float*>(s_red + kFlatCombineThreads);
     float* s_w = s_comb;                           // [n][rows]: first the piece maxima, then the merge weights
     float* s_l = s_comb + (size_t)n * rows;        // [n][rows]: the pieces' sums
     float* s_inv = s_comb + 2 * (size_t)n * rows;  // [rows]
@@ -706,6 +707,44 @@ __global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(
     }
     __syncthreads();
     const int quads = p.d / 4;                     // a thread produces four channels of one row at a time
+    auto store_row = [&](int rr, int c, float4 acc) {
+        const int r = row0 + rr;
+        const float inv = s_inv[rr];
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        const size_t row_out = ((size_t)b * p.R + r / G) * p.Hq + g * G + r % G;
+        uint2 packed;
+        packed.x = pack_bf16x2(acc.x, acc.y);
+        packed.y = pack_bf16x2(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(p.out + row_out * p.d + c) = packed;
+        if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row_out * p.d + c) = acc;
+    };
+    // Few outputs and many pieces (a short batch cut across the whole grid): several threads share an
+    // output, thread group k summing pieces k, k + groups, ... with all its loads in flight at once; the
+    // groups' sums are then added in group order.  The order of the sums is fixed, so results repeat.
+    const int want = rows * quads, groups = (int)blockDim.x / want;
+    if (groups >= 2 && n >= 4) {
+        const int grp = threadIdx.x / want, idx = threadIdx.x % want;
+        const int rr = idx / quads, r = row0 + rr, c = (idx % quads) * 4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (grp < groups) {
+#pragma unroll 4
+            for (int i = grp; i < n; i += groups) {
+                const float4 v = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i) * rows_pad + r) * p.d + c);
+                const float w = s_w[(size_t)i * rows + rr];
+                acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+            }
+            s_red[threadIdx.x] = acc;
+        }
+        __syncthreads();
+        if (grp == 0) {
+            for (int k = 1; k < groups; ++k) {
+                const float4 v = s_red[k * want + idx];
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            store_row(rr, c, acc);
+        }
+        return;
+    }
     for (int idx = threadIdx.x; idx < rows * quads; idx += blockDim.x) {
         const int rr = idx / quads, r = row0 + rr, c = (idx % quads) * 4;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -727,14 +766,7 @@ __global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(
             const float w = s_w[(size_t)i * rows + rr];
             acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
         }
-        const float inv = s_inv[rr];
-        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        const size_t row_out = ((size_t)b * p.R + r / G) * p.Hq + g * G + r % G;
-        uint2 packed;
-        packed.x = pack_bf16x2(acc.x, acc.y);
-        packed.y = pack_bf16x2(acc.z, acc.w);
-        *reinterpret_cast<uint2*>(p.out + row_out * p.d + c) = packed;
-        if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row_out * p.d + c) = acc;
+        store_row(rr, c, acc);
     }
 }
 
@@ -770,10 +802,11 @@ cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtens
         if (row_groups > rows) row_groups = rows;
         const int rows_per_cta = (rows + row_groups - 1) / row_groups;
         row_groups = (rows + rows_per_cta - 1) / rows_per_cta;
-        const size_t comb_smem = (2 * (size_t)ctas + 1) * rows_per_cta * sizeof(float);
+        const size_t comb_smem = (2 * (size_t)ctas + 1) * rows_per_cta * sizeof(float) + kFlatCombineThreads * sizeof(float4);
         e = cudaFuncSetAttribute(attn_flat_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)comb_smem);
         if (e != cudaSuccess) return e;
-        const int threads = rows_per_cta * (p.d / 4) <= 64 ? 64 : (rows_per_cta * (p.d / 4) <= 128 ? 128 : kFlatCombineThreads);
+        // with few outputs per CTA the spare threads share the pieces of an output (see the kernel)
+        const int threads = kFlatCombineThreads;
         e = launch_pdl(attn_flat_combine_kernel, dim3(pairs, row_groups), dim3(threads), comb_smem, stream, p, attn_rows_pad(rows), rows_per_cta);
         *launched = 2;
         return e;
