@@ -49,6 +49,17 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
     const float inv_T = greedy ? 1.f : 1.f / p.T;
     __shared__ Stat row_stat[kMaxRows];
     static_assert(kScanThreads / 32 >= kMaxRows, "one warp per block row");
+    // The drafted tokens, their uniforms and the drafter's probabilities at them are inputs of the step, not
+    // results of the kernel before this one: fetch them while that kernel drains (two dependent cold reads).
+    int x_in = -1;
+    float u_in = 0.f, q_in = 0.f;
+    if (warp == 0 && lane < p.gamma) {
+        x_in = p.draft_tokens[(size_t)b * p.gamma + lane];
+        if (!greedy) {
+            u_in = p.u_accept[(size_t)b * p.gamma + lane];
+            if (!p.q_at_draft && x_in >= 0 && x_in < p.V) q_in = p.draft_probs[((size_t)b * p.gamma + lane) * p.V + x_in];
+        }
+    }
     pdl_wait();
     pdl_trigger();
 
@@ -91,7 +102,7 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
     bool ok = true;
     int x = -1;
     if (lane < p.gamma) {
-        x = p.draft_tokens[(size_t)b * p.gamma + lane];
+        x = x_in;
         if (x < 0 || x >= p.V) {
             set_status(p.dev_status, MASSV_ERR_INVALID_ARG);
             ok = false;
@@ -107,10 +118,10 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
                 }
             } else {
                 zx = p.logits[(size_t)(b * R + lane) * p.V + x];
-                qx = p.draft_probs[((size_t)b * p.gamma + lane) * p.V + x];
+                qx = q_in;
             }
             const float px = expf((zx - row_stat[lane].m) * inv_T) / row_stat[lane].s;
-            const float lhs = p.u_accept[(size_t)b * p.gamma + lane] * qx;
+            const float lhs = u_in * qx;
             ok = lhs < px;
         }
     }
