@@ -315,6 +315,9 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
         }
     }
     pdl_wait();          // everything above overlapped with the tail of the previous kernel
+    // The acceptance kernels behind this one are small: let them become resident now, fetch the inputs that
+    // do not depend on this grid, and wait for it there.
+    pdl_trigger();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -460,7 +463,6 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
 
     tc_fence_before();
     __syncthreads();
-    pdl_trigger();
     // the CTA's statistics: merge the four lane quarters (ascending rows) into one partial slot
     for (int c = threadIdx.x; c < p.n_tile; c += kThreads) {
         const int tok = tok_base + c;
