@@ -201,8 +201,8 @@ static int sample_inverse_cdf(const double *r, int V, double u, double *margin)
  * T > 0  (p = softmax(z/T) passed in `p`, q in `draft_probs`):
  *   draft j (token x = draft_tokens[b,j]) is accepted with probability
  *   min(1, p_j(x)/q_j(x)); with the supplied uniform this is the division-free
- *   test  u_accept[b,j] * q_j(x) < p_j(x), taken in fp32 (the precision in
- *   which the CUDA path takes it).  At the first rejection n the extra token
+ *   test  u_accept[b,j] * q_j(x) < p_j(x), with the product and the comparison
+ *   in double.  At the first rejection n the extra token
  *   is drawn from norm(max(p_n - q_n, 0)); if all gamma are accepted (n =
  *   gamma) it is drawn from p_gamma, the (gamma+1)-th distribution the target
  *   computed.  The draw uses u_sample[b,n].  If the residual has no mass
@@ -239,8 +239,7 @@ void oracle_accept(int B, int gamma, int V, double T, const double *z, const dou
                 double ratio = qj > 0.0f ? pj / (double)qj : (pj > 0.0 ? INFINITY : 0.0);
                 double thr = ratio < 1.0 ? ratio : 1.0;
                 margin_accept[(size_t)b * gamma + j] = fabs((double)u - thr);
-                float lhs = u * qj;                       /* fp32 product, as on the GPU */
-                int ok = lhs < (float)pj;
+                int ok = (double)u * (double)qj < pj;
                 if (!ok) { n = j; break; }
                 out_tokens[(size_t)b * R + j] = x;
             }
