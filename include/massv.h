@@ -371,6 +371,14 @@ typedef struct CUevent_st *massv_event_t;     /* a cudaEvent_t */
 int massv_set_timing_events(massv_event_t lm_head_start, massv_event_t lm_head_stop,
                             massv_event_t attn_start, massv_event_t attn_stop);
 
+/* The same hook, one kernel at a time: `kernel` is one of MASSV_TIMED_*; NULL for both events
+ * switches that kernel's hook off.  MASSV_TIMED_RESIDUAL is the residual / bonus draw of
+ * massv_accept at T > 0 (the one pass over the vocabulary row the extra token is drawn from). */
+#define MASSV_TIMED_LM_HEAD 0
+#define MASSV_TIMED_ATTN 1
+#define MASSV_TIMED_RESIDUAL 2
+int massv_set_kernel_timing(int32_t kernel, massv_event_t start, massv_event_t stop);
+
 #ifdef __cplusplus
 }
 #endif

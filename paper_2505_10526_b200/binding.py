@@ -88,6 +88,8 @@ def _load():
     lib.massv_launch_count.restype = ctypes.c_uint64
     lib.massv_set_timing_events.restype = ctypes.c_int
     lib.massv_set_timing_events.argtypes = [vp, vp, vp, vp]
+    lib.massv_set_kernel_timing.restype = ctypes.c_int
+    lib.massv_set_kernel_timing.argtypes = [ctypes.c_int32, vp, vp]
     return lib
 
 
@@ -135,6 +137,24 @@ def massv_set_timing_events(lm_head=None, attn=None) -> None:
     rc = _lib.massv_set_timing_events(*handles(lm_head), *handles(attn))
     if rc != 0:
         raise MassvError(rc, "massv_set_timing_events")
+
+
+TIMED_LM_HEAD, TIMED_ATTN, TIMED_RESIDUAL = 0, 1, 2
+
+
+def massv_set_kernel_timing(kernel: int, pair=None) -> None:
+    """Record a pair of torch CUDA events around one kernel (TIMED_*) of the following calls on this
+    thread; None switches that kernel's hook off."""
+    if pair is None:
+        a = b = None
+    else:
+        for ev in pair:
+            if not getattr(ev, "cuda_event", 0):
+                ev.record()                 # torch creates the underlying CUDA event lazily
+        a, b = ctypes.c_void_p(pair[0].cuda_event), ctypes.c_void_p(pair[1].cuda_event)
+    rc = _lib.massv_set_kernel_timing(int(kernel), a, b)
+    if rc != 0:
+        raise MassvError(rc, "massv_set_kernel_timing")
 
 
 def massv_strerror(status: int) -> str:

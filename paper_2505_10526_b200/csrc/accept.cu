@@ -548,7 +548,10 @@ cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream) {
     if (launch_pdl(accept_scan_kernel, dim3(p.B), dim3(kScanThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
     count_launches(1);
     if (p.T > 0.f) {
+        const TimingHooks& hooks = timing_hooks();
+        if (hooks.residual_start && cudaEventRecord(hooks.residual_start, stream) != cudaSuccess) return cudaGetLastError();
         if (launch_pdl(residual_sample_kernel, dim3(p.n_chunks, p.B), dim3(kSampleThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+        if (hooks.residual_stop && cudaEventRecord(hooks.residual_stop, stream) != cudaSuccess) return cudaGetLastError();
         count_launches(1);
         if (p.probs_out) {
             const int M = p.B * (p.gamma + 1);

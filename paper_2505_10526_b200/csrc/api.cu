@@ -471,6 +471,18 @@ int massv_set_timing_events(massv_event_t lm_head_start, massv_event_t lm_head_s
     return MASSV_OK;
 }
 
+int massv_set_kernel_timing(int32_t kernel, massv_event_t start, massv_event_t stop) {
+    if ((start == nullptr) != (stop == nullptr)) return MASSV_ERR_INVALID_ARG;
+    TimingHooks& h = timing_hooks();
+    cudaEvent_t a = reinterpret_cast<cudaEvent_t>(start), b = reinterpret_cast<cudaEvent_t>(stop);
+    switch (kernel) {
+        case MASSV_TIMED_LM_HEAD: h.lm_head_start = a; h.lm_head_stop = b; return MASSV_OK;
+        case MASSV_TIMED_ATTN: h.attn_start = a; h.attn_stop = b; return MASSV_OK;
+        case MASSV_TIMED_RESIDUAL: h.residual_start = a; h.residual_stop = b; return MASSV_OK;
+        default: return MASSV_ERR_INVALID_ARG;
+    }
+}
+
 uint64_t massv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

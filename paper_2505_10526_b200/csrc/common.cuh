@@ -78,6 +78,7 @@ struct SeqState {
 // Optional per-thread timing hooks (massv_set_timing_events): events recorded around the dominant kernel of a call.
 struct TimingHooks {
     cudaEvent_t lm_head_start = nullptr, lm_head_stop = nullptr, attn_start = nullptr, attn_stop = nullptr;
+    cudaEvent_t residual_start = nullptr, residual_stop = nullptr;
 };
 TimingHooks& timing_hooks();
 

@@ -8,8 +8,7 @@ three small exchange buffers between ranks (three all-gathers per step, one at t
 * ``run_lockstep`` -- all ranks of a world on ONE device, phase by phase, concatenation in place of the
   all-gather: the single-GPU check of the multi-rank path (no rank's kernel waits on another's).  Its
   "publish" transport uses the library's own all-gather-by-stores kernel (``massv_shard_publish``), the
-  ranks' gathered buffers standing for peer-mapped memory.  ``python -m paper_2505_10526_b200.sharded
-  --config NAME --world W`` runs it on a named workload and prints rank 0's kernel times.
+  ranks' gathered buffers standing for peer-mapped memory.
 
 The phases are a generator's steps: a rank yields the buffer it wants gathered and is resumed with the
 gathered one, so both transports drive the same code.
@@ -136,61 +135,3 @@ class ShardedAccept:
     def run(self, comm, **inputs):
         """One step of this rank against a communicator (every rank of the group calls it)."""
         return drive(self.phases(**inputs), comm)
-
-
-def _main():
-    """All ranks of a world on one GPU, in lockstep, on a named synthetic workload: checks that the ranks
-    agree and prints one JSON line with rank 0's kernel times per phase (medians; the exchanges between
-    the phases are not in them) and the bytes each rank contributes to every exchange."""
-    import argparse
-    import json
-
-    from workloads import generate, get_config
-
-    ap = argparse.ArgumentParser(description=_main.__doc__)
-    ap.add_argument("--config", default="qwen7b_b16_t1")
-    ap.add_argument("--world", type=int, default=4)
-    ap.add_argument("--iters", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--transport", choices=["concat", "publish"], default="publish")
-    a = ap.parse_args()
-    cfg = get_config(a.config)
-    if cfg.vocab % a.world:
-        raise SystemExit("the vocabulary must divide evenly among the ranks")
-    w = generate(cfg, device="cuda", with_attention=False)
-    Vs = cfg.vocab // a.world
-    ranks = [ShardedAccept(cfg.batch, cfg.gamma, cfg.hidden, Vs, cfg.temperature, a.world, r) for r in range(a.world)]
-    inputs = []
-    for r in range(a.world):
-        kw = dict(hidden=w["hidden"], lm_head_shard=w["lm_head"][r * Vs:(r + 1) * Vs].contiguous(),
-                  draft_tokens=w["draft_tokens"])
-        if cfg.temperature > 0:
-            kw.update(draft_probs_shard=w["draft_probs"][:, :, r * Vs:(r + 1) * Vs].contiguous(),
-                      u_accept=w["u_accept"], u_sample=w["u_sample"])
-        inputs.append(kw)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # larger than L2
-    spans = {}
-    for it in range(a.warmup + a.iters):
-        flush.zero_()
-        ranks[0].marks = [] if it >= a.warmup else None
-        res = run_lockstep(ranks, inputs, transport=a.transport)
-        torch.cuda.synchronize()
-        for t, l in res[1:]:
-            assert torch.equal(t, res[0][0]) and torch.equal(l, res[0][1]), "ranks disagree"
-        if ranks[0].marks:
-            ev = dict(ranks[0].marks)
-            for name in ("lm_head", "scan", "pick", "set_token"):
-                if name + ":start" in ev:
-                    spans.setdefault(name, []).append(ev[name + ":start"].elapsed_time(ev[name + ":stop"]))
-    assert all(int(r.dev_status.item()) == 0 for r in ranks)
-    med = {k: round(sorted(v)[len(v) // 2], 4) for k, v in spans.items()}
-    r0 = ranks[0]
-    print(json.dumps(dict(workload=cfg.name, world=a.world, transport=a.transport, shard_vocab=Vs,
-                          rank0_kernel_ms=med, rank0_kernel_ms_total=round(sum(med.values()), 4),
-                          exchange_bytes_per_rank=dict(stats=r0.stats.numel() * 4, masses=r0.masses.numel() * 8,
-                                                       token=r0.token.numel() * 4),
-                          mean_accept_len=float(res[0][1].float().mean()))))
-
-
-if __name__ == "__main__":
-    _main()

@@ -73,55 +73,65 @@ class VerifyStep:
 
     # -- end-to-end step with host buffers ----------------------------------------------
     def host_inputs_like(self, tensors):
-        """Pinned host buffers for the per-step inputs, shaped like ``tensors`` (a dict of name ->
-        tensor): views of ONE pinned allocation, mirrored by ONE device allocation, so that
-        ``run_host`` moves a step's inputs with a single copy however many tensors they are.  The
-        caller writes each step's inputs into the returned views in place."""
-        align = 256
-        layout, off = {}, 0
-        for k, v in tensors.items():
-            nbytes = v.numel() * v.element_size()
-            layout[k] = (off, nbytes, v.dtype, tuple(v.shape))
-            off = (off + nbytes + align - 1) // align * align
-        self._host_blob = torch.empty((max(off, align),), dtype=torch.uint8).pin_memory()
-        self._dev_blob = torch.empty((max(off, align),), dtype=torch.uint8, device=self.device)
-        view = lambda blob: {k: blob[o:o + n].view(dt).view(shape) for k, (o, n, dt, shape) in layout.items()}
-        self._host_views, self._staging = view(self._host_blob), view(self._dev_blob)
-        for k, v in tensors.items():
-            self._host_views[k].copy_(v)
-        self._host_out_blob = torch.empty(self._out_blob.shape, dtype=torch.int32).pin_memory()
-        n_tok = self.B * self.R
-        self._host_out = (self._host_out_blob[:n_tok].view(self.B, self.R), self._host_out_blob[n_tok:])
-        return self._host_views
+        """Pinned host buffers for per-step inputs, shaped like ``tensors`` (a dict of name ->
+        tensor): a ``HostInputs`` dict whose values are views of ONE pinned allocation, mirrored by
+        ONE device allocation, so that ``run_host`` moves a step's inputs with a single copy however
+        many tensors they are.  The caller writes each step's inputs into the returned views in place.
+        Several sets may exist side by side (say, one with and one without the draft distributions)."""
+        return HostInputs(tensors, self.device)
+
+    def _host_result(self):
+        if self._host_out is None:
+            self._host_out_blob = torch.empty(self._out_blob.shape, dtype=torch.int32).pin_memory()
+            n_tok = self.B * self.R
+            self._host_out = (self._host_out_blob[:n_tok].view(self.B, self.R), self._host_out_blob[n_tok:])
+        return self._host_out
 
     def run_host(self, host_inputs, resident, commit=False):
         """One step whose per-step inputs start in pinned host memory and whose result (tokens and
-        accepted lengths) ends in pinned host memory.  ``host_inputs`` are the views returned by
-        ``host_inputs_like`` (one copy up, one copy down) or any dict of pinned tensors (one copy
-        per tensor).  Returns (out_tokens, accept_len) host tensors after synchronising."""
+        accepted lengths) ends in pinned host memory.  ``host_inputs`` is what ``host_inputs_like``
+        returned (one copy up, one copy down) or any dict of pinned tensors (one copy per tensor);
+        ``resident`` holds everything that already lives on the device.  Returns (out_tokens,
+        accept_len) host tensors after synchronising."""
         w = dict(resident)
-        if getattr(self, "_host_views", None) is not None and host_inputs is self._host_views:
-            self._dev_blob.copy_(self._host_blob, non_blocking=True)
-            w.update(self._staging)
+        out = self._host_result()
+        if isinstance(host_inputs, HostInputs):
+            host_inputs.dev_blob.copy_(host_inputs.host_blob, non_blocking=True)
+            w.update(host_inputs.dev_views)
         else:
             if self._staging is None or set(self._staging) != set(host_inputs):
                 self._staging = {k: torch.empty_like(v, device=self.device) for k, v in host_inputs.items()}
-            if self._host_out is None:
-                self._host_out_blob = torch.empty(self._out_blob.shape, dtype=torch.int32).pin_memory()
-                n_tok = self.B * self.R
-                self._host_out = (self._host_out_blob[:n_tok].view(self.B, self.R), self._host_out_blob[n_tok:])
             for k, v in host_inputs.items():
                 self._staging[k].copy_(v, non_blocking=True)
                 w[k] = self._staging[k]
         self.run(w, commit=commit)
         self._host_out_blob.copy_(self._out_blob, non_blocking=True)
         torch.cuda.current_stream().synchronize()
-        return self._host_out
+        return out
 
     def host_bytes_per_step(self, host_inputs):
-        if getattr(self, "_host_views", None) is not None and host_inputs is self._host_views:
-            h2d = self._host_blob.numel()           # the whole staging buffer goes up, padding included
+        if isinstance(host_inputs, HostInputs):
+            h2d = host_inputs.host_blob.numel()     # the whole staging buffer goes up, padding included
         else:
             h2d = sum(v.numel() * v.element_size() for v in host_inputs.values())
         d2h = self.out_tokens.numel() * 4 + self.accept_len.numel() * 4
         return h2d, d2h
+
+
+class HostInputs(dict):
+    """name -> pinned host view; ``host_blob`` / ``dev_blob`` are the two allocations behind the
+    views and ``dev_views`` the device-side tensors of the same names."""
+
+    def __init__(self, tensors, device, align=256):
+        layout, off = {}, 0
+        for k, v in tensors.items():
+            nbytes = v.numel() * v.element_size()
+            layout[k] = (off, nbytes, v.dtype, tuple(v.shape))
+            off = (off + nbytes + align - 1) // align * align
+        self.host_blob = torch.empty((max(off, align),), dtype=torch.uint8).pin_memory()
+        self.dev_blob = torch.empty((max(off, align),), dtype=torch.uint8, device=device)
+        view = lambda blob: {k: blob[o:o + n].view(dt).view(shape) for k, (o, n, dt, shape) in layout.items()}
+        super().__init__(view(self.host_blob))
+        self.dev_views = view(self.dev_blob)
+        for k, v in tensors.items():
+            self[k].copy_(v)

@@ -62,5 +62,16 @@ def compare_accept(ref, tokens, lens, gamma):
     return stats
 
 
+def oracle_attention(w, window=0):
+    """The oracle's append + attention alone on a workload dict (attn_out, lse and the page pools
+    after the append), for cases that compare attention on more sequences than the whole step."""
+    seq = w["seq_lens"].cpu().numpy().astype(np.int32).copy()
+    kp, vp = oracle.bf16_bits(w["k_pages"]).copy(), oracle.bf16_bits(w["v_pages"]).copy()
+    pt = w["page_table"].cpu().numpy().astype(np.int32)
+    oracle.kv_append(oracle.bf16_bits(w["k_new"]), oracle.bf16_bits(w["v_new"]), kp, vp, pt, seq)
+    out, lse = oracle.verify_attn(oracle.bf16_bits(w["q"]), kp, vp, pt, seq, None, window)
+    return dict(attn_out=out, lse=lse, k_pages=kp, v_pages=vp)
+
+
 def oracle_step(w, temperature, want_attention=True):
     return oracle.verify_step(w, temperature, want_attention=want_attention)

@@ -15,7 +15,7 @@ import pytest
 import torch
 
 import oracle
-from parity_util import compare_accept, sub_workload
+from parity_util import compare_accept, oracle_attention, sub_workload
 from workloads import generate, get_config
 
 pytestmark = pytest.mark.gpu
@@ -35,7 +35,7 @@ def _report(entry):
     print(entry)
 
 
-def run_case(name, subset=None, check_determinism=True, cfg=None, window=0, **step_kw):
+def run_case(name, subset=None, check_determinism=True, cfg=None, window=0, attn_subset=None, **step_kw):
     from paper_2505_10526_b200 import VerifyStep
     cfg = cfg or get_config(name)
     w = generate(cfg, device="cuda")
@@ -47,32 +47,40 @@ def run_case(name, subset=None, check_determinism=True, cfg=None, window=0, **st
     assert int(step.dev_status.item()) == 0
 
     idx = list(range(cfg.batch)) if subset is None else subset
+    # attn_subset: sequences whose attention (and appended cache bytes) are compared, when that is a
+    # larger set than the one the whole step is compared on ("all": the whole batch)
+    idx_attn = idx if attn_subset is None else (list(range(cfg.batch)) if attn_subset == "all" else attn_subset)
     # the oracle sees the inputs as they were before the step
     w_ref = dict(w)
     w_ref["k_pages"], w_ref["v_pages"] = pools_before
     w_ref["seq_lens"] = seq_before
-    ref = oracle.verify_step(sub_workload(w_ref, idx), cfg.temperature, window=window)
+    ref = oracle.verify_step(sub_workload(w_ref, idx), cfg.temperature, window=window, want_attention=idx_attn == idx)
+    if idx_attn != idx:
+        ref.update(oracle_attention(sub_workload(w_ref, idx_attn), window=window))
     R, V = cfg.rows, cfg.vocab
     sel = torch.as_tensor(idx, device="cuda")
+    sel_attn = torch.as_tensor(idx_attn, device="cuda")
 
-    entry = dict(config=name, sequences=len(idx))
+    entry = dict(config=name or cfg.name, sequences=len(idx), sequences_attention=len(idx_attn), batch=cfg.batch)
     # -- appended cache bytes: every position < L + R of the checked sequences, bit-exact
     kp, vp = oracle.bf16_bits(w["k_pages"]), oracle.bf16_bits(w["v_pages"])
     pt = w["page_table"].cpu().numpy()
-    for i, b in enumerate(idx):
+    for i, b in enumerate(idx_attn):
         n = int(seq_before[b]) + R
         pages = pt[b, :(n + 15) // 16]
         assert np.array_equal(kp[pages], ref["k_pages"][pages]) and np.array_equal(vp[pages], ref["v_pages"][pages])
     # pages of other sequences and unmapped pages are untouched unless they hold block slots
-    if subset is None:
+    if len(idx_attn) == cfg.batch:
         assert np.array_equal(kp, ref["k_pages"]) and np.array_equal(vp, ref["v_pages"])
+    del kp, vp
     # -- attention
-    o32 = step.attn_out_f32.index_select(0, sel).cpu().double().numpy()
-    o16 = step.attn_out.index_select(0, sel).cpu().double().numpy()
-    lse = step.lse.index_select(0, sel).cpu().double().numpy()
+    o32 = step.attn_out_f32.index_select(0, sel_attn).cpu().double().numpy()
+    o16 = step.attn_out.index_select(0, sel_attn).cpu().double().numpy()
+    lse = step.lse.index_select(0, sel_attn).cpu().double().numpy()
     entry["attn_err_f32"] = float(np.abs(o32 - ref["attn_out"]).max())
     entry["attn_err_bf16"] = float(np.abs(o16 - ref["attn_out"]).max())
     entry["lse_err"] = float(np.abs(lse - ref["lse"]).max())
+    ref.pop("k_pages", None); ref.pop("v_pages", None)
     # -- logits / probabilities
     z = step.logits.index_select(0, sel).cpu().double().numpy().reshape(-1, V)
     entry["logit_err"] = float(np.abs(z - ref["logits"]).max())
@@ -127,14 +135,27 @@ def test_qwen_batch16_sampling_full_parity(name):
         assert 1.5 < e["mean_accept_len"] < 3.6
 
 
-def test_gemma_batch32_sampled_sequences():
-    run_case("gemma12b_b32_t1", subset=[0, 7, 19, 31], check_determinism=False)
+def test_gemma_batch32_full_parity():
+    """Config 4, every one of the 32 sequences, the whole step."""
+    e = run_case("gemma12b_b32_t1")
+    assert e["sequences"] == e["batch"] == 32
 
 
-@pytest.mark.parametrize("gamma", [3, 5, 7])
-@pytest.mark.parametrize("t", [0, 1])
-def test_long_context_sweep_sampled_sequences(gamma, t):
-    run_case(f"qwen7b_long_g{gamma}_t{t}", subset=[0, 33, 63], check_determinism=False)
+@pytest.mark.parametrize("name", ["qwen7b_long_g5_t1", "qwen7b_long_g7_t0"])
+def test_long_context_whole_batch_whole_step(name):
+    """Config 5, one point per temperature: all 64 sequences through the whole step (the flat attention
+    schedule cuts (sequence, head) pairs at places that depend on the whole batch, so every sequence is
+    compared, not a sample)."""
+    e = run_case(name)
+    assert e["sequences"] == e["sequences_attention"] == e["batch"] == 64
+
+
+@pytest.mark.parametrize("name", ["qwen7b_long_g3_t0", "qwen7b_long_g3_t1", "qwen7b_long_g5_t0", "qwen7b_long_g7_t1"])
+def test_long_context_whole_batch_attention(name):
+    """The other config-5 points: attention and appended cache bytes for all 64 sequences, the LM head
+    and acceptance on sampled sequences."""
+    e = run_case(name, subset=[0, 33, 63], attn_subset="all", check_determinism=False)
+    assert e["sequences_attention"] == e["batch"] == 64
 
 
 def test_rollback_then_redraft_matches_a_fresh_step():
