@@ -10,6 +10,7 @@
 //   kv_commit_kernel        advance the committed cache lengths.
 // All reductions run in a fixed order, so results are bit-identical run to run.
 #include "kernels.cuh"
+#include "ptx.cuh"
 
 namespace massv {
 
@@ -19,6 +20,10 @@ constexpr int kScanThreads = 256;
 constexpr int kScanBatch = 6;     // partial slots a lane loads before merging (192 slots = one batch)
 constexpr int kSampleThreads = 256;
 constexpr int kPerThread = kResidualChunk / kSampleThreads;   // 16 contiguous entries per thread
+constexpr int kResidualStages = 3; // ring entries (32 KB each: the chunk's logits and the drafter's probabilities)
+constexpr int kResidualThreads = kSampleThreads + 32;   // eight consumer warps and the producer warp
+constexpr int kResidualCtasPerSm = 2;
+constexpr int kResidualSeqCache = 8; // sequences whose scan results a CTA keeps in shared memory
 constexpr int kWalkChunks = 512;  // chunk masses staged in shared memory for the walk (vocabularies up to 2M entries)
 static_assert(kPerThread == 16, "chunk layout");
 
@@ -145,38 +150,75 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
     }
 }
 
-// Masses of the 16 entries this thread owns in chunk c of the sampled row.
-__device__ __forceinline__ void chunk_masses(const AcceptParams& p, int b, const SeqState& st, int use_q, int c,
-                                             float inv_T, float (&r)[kPerThread]) {
-    const int R = p.gamma + 1;
-    const int v0 = c * kResidualChunk + threadIdx.x * kPerThread;
-    const float* z = p.logits + (size_t)(b * R + st.n) * p.V;
-    const float* q = use_q ? p.draft_probs + ((size_t)b * p.gamma + st.n) * p.V : nullptr;
+// A chunk of the sampled row is 4096 vocabulary entries = 1024 groups of four.  Thread t owns groups
+// t, t + 256, t + 512, t + 768 (so that a warp touches consecutive 16-byte words, in shared memory as
+// in global memory); r[4 j + e] is entry e of group t + 256 j.  Vocabulary order inside the chunk is
+// therefore (j, t, e).
+// Barrier among warps 0-7 (the kernels' 256 arithmetic threads; a ninth warp, where there is one, stays out).
+__device__ __forceinline__ void bar_sync_consumers() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+
+// p(v) = exp((z_v - max) / T) / sum, evaluated as 2^(z_v a + bias) with a = log2(e) / T and
+// bias = -max a + log2(1 / sum): one multiply-add into the exponential unit.
+struct RowCtx {
+    float a, bias;
+    __device__ RowCtx(const SeqState& st, float inv_T) {
+        a = inv_T * 1.4426950408889634f;
+        bias = fmaf(-st.row_max, a, log2f(st.inv_sum));
+    }
+    __device__ __forceinline__ float prob(float z) const { return exp2f(fmaf(z, a, bias)); }
+};
+__device__ __forceinline__ void masses_of(const float4 (&zz)[4], const float4 (&qq)[4], bool use_q, int valid, const RowCtx& rc,
+                                          float (&r)[kPerThread]) {
 #pragma unroll
-    for (int g = 0; g < kPerThread; g += 4) {
-        const int v = v0 + g;
-        float zz[4] = {0.f, 0.f, 0.f, 0.f}, qq[4] = {0.f, 0.f, 0.f, 0.f};
-        if (v + 3 < p.V) {
-            const float4 a = *reinterpret_cast<const float4*>(z + v);
-            zz[0] = a.x; zz[1] = a.y; zz[2] = a.z; zz[3] = a.w;
-            if (q) {
-                const float4 d = __ldg(reinterpret_cast<const float4*>(q + v));
-                qq[0] = d.x; qq[1] = d.y; qq[2] = d.z; qq[3] = d.w;
-            }
-        } else {
-            for (int e = 0; e < 4; ++e)
-                if (v + e < p.V) { zz[e] = z[v + e]; if (q) qq[e] = q[v + e]; }
-        }
+    for (int j = 0; j < 4; ++j) {
+        const int e0 = 4 * ((int)threadIdx.x + kSampleThreads * j);       // first entry of the group inside the chunk
+        const float z[4] = {zz[j].x, zz[j].y, zz[j].z, zz[j].w}, q[4] = {qq[j].x, qq[j].y, qq[j].z, qq[j].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             float m = 0.f;
-            if (v + e < p.V) {
-                const float pv = expf((zz[e] - st.row_max) * inv_T) * st.inv_sum;
-                m = q ? fmaxf(pv - qq[e], 0.f) : pv;
+            if (e0 + e < valid) {
+                const float pv = rc.prob(z[e]);
+                m = use_q ? fmaxf(pv - q[e], 0.f) : pv;
             }
-            r[g + e] = m;
+            r[4 * j + e] = m;
         }
     }
+}
+// The same from global memory: z and q point at the chunk's first entry; `valid` entries exist (a multiple of 4).
+__device__ __forceinline__ void chunk_masses_global(const float* z, const float* q, int valid, const RowCtx& rc,
+                                                    float (&r)[kPerThread]) {
+    float4 zz[4], qq[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int e0 = 4 * ((int)threadIdx.x + kSampleThreads * j);
+        zz[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        qq[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e0 < valid) {
+            zz[j] = *reinterpret_cast<const float4*>(z + e0);
+            if (q) qq[j] = __ldg(reinterpret_cast<const float4*>(q + e0));
+        }
+    }
+    masses_of(zz, qq, q != nullptr, valid, rc, r);
+}
+// Sum of the thread's 16 masses in (j, e) order, in double.
+__device__ __forceinline__ double local_mass(const float (&r)[kPerThread]) {
+    double s = 0.0;
+#pragma unroll
+    for (int i = 0; i < kPerThread; ++i) s += (double)r[i];
+    return s;
+}
+// Block-wide sum in a fixed order (butterfly inside a warp: both partners form the same sum; warps in
+// order).  Every thread receives it.  Two barriers.
+__device__ __forceinline__ double block_total(double x, double* smem_warp) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    if ((threadIdx.x & 31) == 0) smem_warp[threadIdx.x >> 5] = x;
+    bar_sync_consumers();
+    double tot = 0.0;
+#pragma unroll
+    for (int w = 0; w < kSampleThreads / 32; ++w) tot += smem_warp[w];
+    bar_sync_consumers();
+    return tot;
 }
 
 // Block-wide exclusive prefix of one double per thread, in thread order; *total gets the sum.
@@ -189,59 +231,73 @@ __device__ __forceinline__ double block_exclusive_scan(double x, double* smem_wa
         if (lane >= o) incl += y;
     }
     if (lane == 31) smem_warp[warp] = incl;
-    __syncthreads();
+    bar_sync_consumers();
     double base = 0.0, tot = 0.0;
     for (int w = 0; w < kSampleThreads / 32; ++w) {
         const double s = smem_warp[w];
         if (w < warp) base += s;
         tot += s;
     }
-    __syncthreads();
+    bar_sync_consumers();
     *total = tot;
     return base + incl - x;
 }
 
-// grid (n_chunks, B).  Every CTA stores its chunk's mass; the CTA that arrives
-// last for a sequence walks the chunk masses and then the winning chunk.
-__global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptParams p) {
-    const int c = blockIdx.x, b = blockIdx.y, t = threadIdx.x;
-    const int R = p.gamma + 1;
-    const float inv_T = 1.f / p.T;
-    pdl_wait();
-    pdl_trigger();
-    const SeqState st = p.seq_state[b];
-    __shared__ double warp_sums[kSampleThreads / 32];
-    __shared__ int s_flag;
-    __shared__ int s_pick[2];
-    __shared__ double s_base[2];
-
-    float r[kPerThread];
-    chunk_masses(p, b, st, st.use_q, c, inv_T, r);
-    double local = 0.0;
+// Inside the chunk that holds the target: the first entry (in vocabulary order) whose running mass
+// exceeds `target`, starting from `base`, and the last entry with positive mass.  r as produced by
+// masses_of.  Results through s_first / s_last (shared), valid after the call for every thread.
+__device__ __forceinline__ void pick_in_chunk(const float (&r)[kPerThread], int chunk_first_entry, double base, double target,
+                                              double* smem_warp, int* s_first, int* s_last) {
+    const int t = threadIdx.x;
+    if (t == 0) { *s_first = 0x7fffffff; *s_last = -1; }
+    int first = 0x7fffffff, last = -1;
+    double run_base = base;
 #pragma unroll
-    for (int e = 0; e < kPerThread; ++e) local += (double)r[e];
-    double total;
-    block_exclusive_scan(local, warp_sums, &total);
-    double* sums = p.chunk_sums + (size_t)b * p.n_chunks;
-    if (t == 0) {
-        sums[c] = total;
-        __threadfence();
-        const unsigned prev = atomicAdd(&p.counters[b], 1u);
-        s_flag = (prev == (unsigned)p.n_chunks - 1u);
+    for (int j = 0; j < 4; ++j) {            // quarter j of the chunk: groups 256 j .. 256 j + 255, one per thread
+        const double g = ((double)r[4 * j] + (double)r[4 * j + 1]) + ((double)r[4 * j + 2] + (double)r[4 * j + 3]);
+        double quarter;
+        double run = run_base + block_exclusive_scan(g, smem_warp, &quarter);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            run += (double)r[4 * j + e];
+            if (r[4 * j + e] > 0.f) {
+                const int v = chunk_first_entry + 4 * (t + kSampleThreads * j) + e;
+                last = v;
+                if (first == 0x7fffffff && run > target) first = v;
+            }
+        }
+        run_base += quarter;
     }
-    __syncthreads();
-    if (!s_flag) return;
-    __threadfence();
+    bar_sync_consumers();
+    atomicMin(s_first, first);
+    atomicMax(s_last, last);
+    bar_sync_consumers();
+}
 
-    // The walk over the chunk masses is sequential (fixed summation order) but its loads need not be:
-    // the CTA fetches the masses the other CTAs wrote (L2, bypassing L1) into shared memory at once.
-    __shared__ double s_sums[kWalkChunks];
+__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(smem_u32(dst)),
+        "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+
+// The sequential part of the draw for one sequence, by the 256 threads of warps 0-7: walk the chunk masses
+// (fixed summation order), then find the token inside the winning chunk.
+__device__ void draw_from_chunk_masses(const AcceptParams& p, int b, const SeqState& st, float inv_T, double* warp_sums, double* s_sums,
+                                       int* s_pick, double* s_base, int* s_first, int* s_last) {
+    const int t = threadIdx.x, R = p.gamma + 1;
+    const RowCtx rc(st, inv_T);
+    double* sums = p.chunk_sums + (size_t)b * p.n_chunks;
+    // The walk is sequential but its loads need not be: the masses the other CTAs wrote come from L2
+    // (bypassing L1) into shared memory at once.
     const bool staged = p.n_chunks <= kWalkChunks;
+    const float* z_row = p.logits + (size_t)(b * R + st.n) * p.V;
+    const float* q_row = p.draft_probs ? p.draft_probs + ((size_t)b * p.gamma + st.n) * p.V : nullptr;
     int use_q = st.use_q;
     for (int attempt = 0; attempt < 2; ++attempt) {
         if (staged) {
             for (int i = t; i < p.n_chunks; i += kSampleThreads) s_sums[i] = __ldcg(sums + i);
-            __syncthreads();
+            bar_sync_consumers();
         }
         if (t == 0) {
             double tot = 0.0;
@@ -250,86 +306,198 @@ __global__ void __launch_bounds__(kSampleThreads) residual_sample_kernel(AcceptP
             int pick = -1, last_pos = -1;
             double cum = 0.0, base = 0.0;
             for (int i = 0; i < p.n_chunks; ++i) {
-                const double s = staged ? s_sums[i] : ((volatile double*)sums)[i];
-                if (s > 0.0) last_pos = i;
-                if (pick < 0 && s > 0.0 && cum + s > target) { pick = i; base = cum; }
-                cum += s;
+                const double sm = staged ? s_sums[i] : ((volatile double*)sums)[i];
+                if (sm > 0.0) last_pos = i;
+                if (pick < 0 && sm > 0.0 && cum + sm > target) { pick = i; base = cum; }
+                cum += sm;
             }
             s_pick[0] = tot > 0.0 ? (pick >= 0 ? pick : last_pos) : -1;
             s_pick[1] = (pick < 0);        // rounding pushed the target past the end: take the last positive entry
             s_base[0] = base;
             s_base[1] = target;
         }
-        __syncthreads();
+        bar_sync_consumers();
         if (s_pick[0] >= 0 || !use_q) break;
         // The residual has no mass (p == q on this row): draw from p instead.
         use_q = 0;
         for (int cc = 0; cc < p.n_chunks; ++cc) {
-            chunk_masses(p, b, st, 0, cc, inv_T, r);
-            double loc = 0.0;
-#pragma unroll
-            for (int e = 0; e < kPerThread; ++e) loc += (double)r[e];
-            double tt;
-            block_exclusive_scan(loc, warp_sums, &tt);
+            float rr[kPerThread];
+            chunk_masses_global(z_row + (size_t)cc * kResidualChunk, nullptr, min(kResidualChunk, p.V - cc * kResidualChunk), rc, rr);
+            const double tt = block_total(local_mass(rr), warp_sums);
             if (t == 0) sums[cc] = tt;
         }
         __threadfence();       // this CTA reads the new masses back through L2 on the second attempt
-        __syncthreads();
+        bar_sync_consumers();
     }
     const int pick = s_pick[0];
     int32_t* tok_out = p.out_tokens + (size_t)b * R + st.n;
     if (pick < 0) {                        // no mass at all (cannot happen for a softmax row)
         if (t == 0) { *tok_out = 0; set_status(p.dev_status, MASSV_ERR_INVALID_ARG); }
-        return;
+    } else {
+        const bool take_last = s_pick[1] != 0;
+        float rr[kPerThread];
+        chunk_masses_global(z_row + (size_t)pick * kResidualChunk, use_q ? q_row + (size_t)pick * kResidualChunk : nullptr,
+                            min(kResidualChunk, p.V - pick * kResidualChunk), rc, rr);
+        pick_in_chunk(rr, pick * kResidualChunk, s_base[0], s_base[1], warp_sums, s_first, s_last);
+        if (t == 0) *tok_out = (!take_last && *s_first != 0x7fffffff) ? *s_first : *s_last;
     }
-    const bool take_last = s_pick[1] != 0;
-    const double base = s_base[0], target = s_base[1];
-    chunk_masses(p, b, st, use_q, pick, inv_T, r);
-    double loc = 0.0;
+    bar_sync_consumers();          // the shared pick state may be reused for this CTA's next sequence
+}
+
+// T > 0: the extra token of every sequence, one pass over the single row it is drawn from.  Work item =
+// (sequence, 4096-entry chunk); a persistent grid of one wave deals the items out in contiguous runs.
+// Warp 8 is the producer: it keeps a ring of items filled with bulk copies (the chunk of the row's logits
+// and, after a rejection, of the drafter's distribution: two contiguous 16 KB runs), so the bytes in flight
+// do not depend on registers.  Warps 0-7 are consumers that never wait for one another: each turns its
+// eighth of a landed item into masses, adds them up in double (lane sums, then a butterfly: a fixed order)
+// and hands its partial sum back with the stage; the producer adds the eight partials in warp order,
+// stores the chunk's mass and counts the sequence's chunks.  The CTA that completes a sequence's last
+// chunk makes the sequential part of the draw once its own items are done.
+__global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual_sample_kernel(AcceptParams p) {
+    extern __shared__ __align__(128) uint8_t res_smem[];
+    __shared__ __align__(8) uint64_t full_bar[kResidualStages];     // the item's bytes have landed
+    __shared__ __align__(8) uint64_t done_bar[kResidualStages];     // the eight consumer warps are done with the stage
+    __shared__ double s_part[kResidualStages][kSampleThreads / 32];
+    __shared__ double warp_sums[kSampleThreads / 32];
+    __shared__ double s_sums[kWalkChunks];
+    __shared__ SeqState s_state[kResidualSeqCache];
+    __shared__ int s_pending[kResidualSeqCache], s_n_pending;
+    __shared__ int s_abort;
+    __shared__ int s_pick[2];
+    __shared__ double s_base[2];
+    __shared__ int s_first, s_last;
+
+    const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+    const int R = p.gamma + 1;
+    const float inv_T = 1.f / p.T;
+    const long total_items = (long)p.B * p.n_chunks;
+    const int i0 = (int)((long)blockIdx.x * total_items / gridDim.x), i1 = (int)((long)(blockIdx.x + 1) * total_items / gridDim.x);
+    const int n_items = i1 - i0;
+    const int b_lo = i0 / p.n_chunks;
+    if (t == 0) {
+        for (int s = 0; s < kResidualStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&done_bar[s], kSampleThreads / 32); }
+        s_abort = 0;
+        s_n_pending = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    pdl_wait();
+    pdl_trigger();
+    if (n_items <= 0) return;
+    {
+        const int n_seq = (i1 - 1) / p.n_chunks - b_lo + 1;
+        if (t < min(n_seq, kResidualSeqCache)) s_state[t] = p.seq_state[b_lo + t];
+    }
+    __syncthreads();
+    auto state_of = [&](int b) -> SeqState { return b - b_lo < kResidualSeqCache ? s_state[b - b_lo] : p.seq_state[b]; };
+    volatile int* abort_ptr = &s_abort;
+    constexpr int kStageBytes = 2 * kResidualChunk * 4;
+
+    if (warp == kSampleThreads / 32) {
+        // ------------------------------------------------ producer
+        if (lane == 0) {
+            uint64_t policy;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+            int run_cnt = 0;               // chunks of the current sequence finished since this CTA's last arrival
+            bool ok = true;
+            for (int k = 0; k < n_items + kResidualStages && ok; ++k) {
+                const int kd = k - kResidualStages;        // the item whose stage is about to be refilled
+                if (kd >= 0) {
+                    const int item = i0 + kd, b = item / p.n_chunks, c = item % p.n_chunks, s = kd % kResidualStages;
+                    if (!mbar_wait(&done_bar[s], ((uint32_t)(kd / kResidualStages)) & 1u, abort_ptr)) { ok = false; break; }
+                    double total = 0.0;
 #pragma unroll
-    for (int e = 0; e < kPerThread; ++e) loc += (double)r[e];
-    double tt;
-    double run = base + block_exclusive_scan(loc, warp_sums, &tt);
-    int first = 0x7fffffff, last = -1;
+                    for (int w = 0; w < kSampleThreads / 32; ++w) total += s_part[s][w];
+                    p.chunk_sums[(size_t)b * p.n_chunks + c] = total;
+                    ++run_cnt;
+                    if (kd + 1 == n_items || (item + 1) / p.n_chunks != b) {      // this CTA's last chunk of sequence b
+                        __threadfence();
+                        const unsigned prev = atomicAdd(&p.counters[b], (unsigned)run_cnt);
+                        if (prev + (unsigned)run_cnt == (unsigned)p.n_chunks) {
+                            // every chunk of b is in: the draw is this CTA's (its slot in the list is free: a CTA
+                            // completes at most one sequence per sequence it holds items of)
+                            if (s_n_pending < kResidualSeqCache) s_pending[s_n_pending++] = b;
+                            else set_status(p.dev_status, MASSV_ERR_UNSUPPORTED);
+                        }
+                        run_cnt = 0;
+                    }
+                }
+                if (k < n_items) {
+                    const int item = i0 + k, b = item / p.n_chunks, c = item % p.n_chunks, s = k % kResidualStages;
+                    const SeqState st = state_of(b);
+                    const uint32_t bytes = (uint32_t)min(kResidualChunk, p.V - c * kResidualChunk) * 4u;
+                    uint8_t* dst = res_smem + (size_t)s * kStageBytes;
+                    mbar_expect_tx(&full_bar[s], st.use_q ? 2 * bytes : bytes);
+                    bulk_load_1d(dst, p.logits + (size_t)(b * R + st.n) * p.V + (size_t)c * kResidualChunk, bytes, &full_bar[s], policy);
+                    if (st.use_q)
+                        bulk_load_1d(dst + kResidualChunk * 4, p.draft_probs + ((size_t)b * p.gamma + st.n) * p.V + (size_t)c * kResidualChunk,
+                                     bytes, &full_bar[s], policy);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------ consumers: warp w owns groups 128 w .. 128 w + 127 of the chunk
+        for (int k = 0; k < n_items; ++k) {
+            const int item = i0 + k, b = item / p.n_chunks, c = item % p.n_chunks, s = k % kResidualStages;
+            const SeqState st = state_of(b);
+            const RowCtx rc(st, inv_T);
+            const int valid = min(kResidualChunk, p.V - c * kResidualChunk);
+            if (!mbar_wait_warp(&full_bar[s], ((uint32_t)(k / kResidualStages)) & 1u, abort_ptr)) break;
+            const float4* zs = reinterpret_cast<const float4*>(res_smem + (size_t)s * kStageBytes);
+            const float4* qs = zs + kResidualChunk / 4;
+            double acc[4];
 #pragma unroll
-    for (int e = 0; e < kPerThread; ++e) {
-        run += (double)r[e];
-        if (r[e] > 0.f) {
-            const int v = pick * kResidualChunk + t * kPerThread + e;
-            last = v;
-            if (first == 0x7fffffff && run > target) first = v;
+            for (int i = 0; i < 4; ++i) {
+                const int g = warp * 128 + i * 32 + lane;          // group of four entries
+                const float4 zv = zs[g];
+                float m[4] = {rc.prob(zv.x), rc.prob(zv.y), rc.prob(zv.z), rc.prob(zv.w)};
+                if (st.use_q) {
+                    const float4 qv = qs[g];
+                    m[0] = fmaxf(m[0] - qv.x, 0.f); m[1] = fmaxf(m[1] - qv.y, 0.f);
+                    m[2] = fmaxf(m[2] - qv.z, 0.f); m[3] = fmaxf(m[3] - qv.w, 0.f);
+                }
+                if (4 * g >= valid) { m[0] = 0.f; m[1] = 0.f; m[2] = 0.f; m[3] = 0.f; }     // past the end of the vocabulary (V % 4 == 0)
+                acc[i] = ((double)m[0] + (double)m[1]) + ((double)m[2] + (double)m[3]);
+            }
+            double x = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if (lane == 0) {
+                s_part[s][warp] = x;
+                mbar_arrive(&done_bar[s]);         // release: the partial sum is visible to the producer's wait
+            }
+            __syncwarp();
         }
     }
-    __shared__ int s_first, s_last;
-    if (t == 0) { s_first = 0x7fffffff; s_last = -1; }
     __syncthreads();
-    atomicMin(&s_first, first);
-    atomicMax(&s_last, last);
-    __syncthreads();
-    if (t == 0) *tok_out = (!take_last && s_first != 0x7fffffff) ? s_first : s_last;
+    if (*abort_ptr) {
+        // a copy never signalled: report it, and give copies that may still be in flight time to land
+        if (t == 0) {
+            set_status(p.dev_status, MASSV_ERR_TIMEOUT);
+            for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        }
+        __syncthreads();
+        return;
+    }
+    if (warp == kSampleThreads / 32) return;
+    const int n_pending = s_n_pending;
+    for (int i = 0; i < n_pending; ++i) {
+        __threadfence();           // the other CTAs' chunk masses, counted before this CTA's arrival
+        const int b = s_pending[i];
+        draw_from_chunk_masses(p, b, state_of(b), inv_T, warp_sums, s_sums, s_pick, s_base, &s_first, &s_last);
+    }
 }
 
 // ---------------------------------------------------------------- vocabulary shards
 // The same arithmetic with the vocabulary cut into contiguous shards, one per rank: a shard sees Vs
 // columns of the logits and of q.  Chunks are counted inside the shard; ranks in order are vocabulary order.
 
-// Masses of the 16 entries this thread owns in chunk c of the sampled row of a shard.
+// Masses of the 16 entries this thread owns in chunk c of the sampled row of a shard (same layout as above).
 __device__ __forceinline__ void shard_chunk_masses(const ShardParams& p, int b, const SeqState& st, int use_q, int c,
                                                    float inv_T, float (&r)[kPerThread]) {
     const int R = p.gamma + 1;
-    const int v0 = c * kResidualChunk + threadIdx.x * kPerThread;
-    const float* z = p.logits + (size_t)(b * R + st.n) * p.Vs;
-    const float* q = use_q ? p.draft_probs + ((size_t)b * p.gamma + st.n) * p.Vs : nullptr;
-#pragma unroll
-    for (int e = 0; e < kPerThread; ++e) {
-        const int v = v0 + e;
-        float m = 0.f;
-        if (v < p.Vs) {
-            const float pv = expf((z[v] - st.row_max) * inv_T) * st.inv_sum;
-            m = q ? fmaxf(pv - q[v], 0.f) : pv;
-        }
-        r[e] = m;
-    }
+    const float* z = p.logits + (size_t)(b * R + st.n) * p.Vs + (size_t)c * kResidualChunk;
+    const float* q = use_q ? p.draft_probs + ((size_t)b * p.gamma + st.n) * p.Vs + (size_t)c * kResidualChunk : nullptr;
+    chunk_masses_global(z, q, min(kResidualChunk, p.Vs - c * kResidualChunk), RowCtx(st, inv_T), r);
 }
 
 // Logit and drafter probability at each drafted token this shard owns (-inf elsewhere: a maximum
@@ -359,11 +527,7 @@ __global__ void __launch_bounds__(kSampleThreads) shard_masses_kernel(ShardParam
         // the residual has no mass anywhere)
         const int use_q = pass == 0 ? st.use_q : 0;
         shard_chunk_masses(p, b, st, use_q, c, inv_T, r);
-        double local = 0.0;
-#pragma unroll
-        for (int e = 0; e < kPerThread; ++e) local += (double)r[e];
-        double total;
-        block_exclusive_scan(local, warp_sums, &total);
+        const double total = block_total(local_mass(r), warp_sums);
         if (t == 0) (pass == 0 ? p.sums_res : p.sums_p)[(size_t)b * p.n_chunks + c] = total;
         if (pass == 0 && !st.use_q) {          // the two passes coincide
             if (t == 0) p.sums_p[(size_t)b * p.n_chunks + c] = total;
@@ -433,26 +597,7 @@ __global__ void __launch_bounds__(kSampleThreads) shard_pick_kernel(ShardParams 
     const double base = s_base[0], target = s_base[1];
     float r[kPerThread];
     shard_chunk_masses(p, b, st, use_q, c, inv_T, r);
-    double loc = 0.0;
-#pragma unroll
-    for (int e = 0; e < kPerThread; ++e) loc += (double)r[e];
-    double tt;
-    double run = base + block_exclusive_scan(loc, warp_sums, &tt);
-    int first = 0x7fffffff, last = -1;
-#pragma unroll
-    for (int e = 0; e < kPerThread; ++e) {
-        run += (double)r[e];
-        if (r[e] > 0.f) {
-            const int v = c * kResidualChunk + t * kPerThread + e;
-            last = v;
-            if (first == 0x7fffffff && run > target) first = v;
-        }
-    }
-    if (t == 0) { s_first = 0x7fffffff; s_last = -1; }
-    __syncthreads();
-    atomicMin(&s_first, first);
-    atomicMax(&s_last, last);
-    __syncthreads();
+    pick_in_chunk(r, c * kResidualChunk, base, target, warp_sums, &s_first, &s_last);
     if (t == 0) p.token_out[b] = p.vocab_offset + ((!take_last && s_first != 0x7fffffff) ? s_first : s_last);
 }
 
@@ -550,7 +695,11 @@ cudaError_t launch_accept(const AcceptParams& p, cudaStream_t stream) {
     if (p.T > 0.f) {
         const TimingHooks& hooks = timing_hooks();
         if (hooks.residual_start && cudaEventRecord(hooks.residual_start, stream) != cudaSuccess) return cudaGetLastError();
-        if (launch_pdl(residual_sample_kernel, dim3(p.n_chunks, p.B), dim3(kSampleThreads), 0, stream, p) != cudaSuccess) return cudaGetLastError();
+        const size_t ring = (size_t)kResidualStages * 2 * kResidualChunk * sizeof(float);
+        if (cudaFuncSetAttribute(residual_sample_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring) != cudaSuccess) return cudaGetLastError();
+        const long items = (long)p.B * p.n_chunks;
+        const long wave = (long)kResidualCtasPerSm * device_sm_count();       // one wave of resident CTAs
+        if (launch_pdl(residual_sample_kernel, dim3((unsigned)(items < wave ? items : wave)), dim3(kResidualThreads), ring, stream, p) != cudaSuccess) return cudaGetLastError();
         if (hooks.residual_stop && cudaEventRecord(hooks.residual_stop, stream) != cudaSuccess) return cudaGetLastError();
         count_launches(1);
         if (p.probs_out) {

@@ -85,6 +85,14 @@ TimingHooks& timing_hooks();
 // Host-side tally of kernel launches (see massv_launch_count).
 void count_launches(int n);
 
+// Multiprocessors of the current device (148 on B200).
+inline int device_sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+        n = 148;
+    return n;
+}
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace massv
