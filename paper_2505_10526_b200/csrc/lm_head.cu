@@ -51,6 +51,8 @@ struct UmmaParams {
     int32_t* part_idx;
     int32_t* dev_status;
     int idx_offset;      // added to the argmax indices that leave the kernel
+    int n_bands = 0;     // duo kernel: 256-row vocabulary bands in all
+    int split_rem = 0;   // duo kernel: bands left over after tiles_per_group per pair, each cut in two half-tiles (one sub-tile each)
 };
 
 // ---- CTA pairs (cta_group::2): two CTAs of a cluster act as one 256-row MMA.  Each loads its own
@@ -188,6 +190,25 @@ __device__ __forceinline__ void transposed_sum(float (&v)[C], int lane) {
         } else {
             v[0] += __shfl_xor_sync(0xffffffffu, v[0], offset);
         }
+    }
+}
+
+// The same exchange pattern for maxima: on return lane l holds the maximum of column l over the 32 lanes.
+__device__ __forceinline__ void transposed_max(float (&v)[32], int lane) {
+    int n = 32;
+#pragma unroll
+    for (int offset = 16; offset >= 1; offset >>= 1) {
+        const int half = n / 2;
+        const bool upper = (lane & offset) != 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            if (i < half) {
+                const float send = upper ? v[i] : v[i + half];
+                const float keep = upper ? v[i + half] : v[i];
+                v[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, offset));
+            }
+        }
+        n = half;
     }
 }
 
@@ -489,6 +510,304 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
     if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
 }
 
+// 64 accumulator columns of this thread's lane (vocabulary row) in one load.
+__device__ __forceinline__ void tmem_load64(uint32_t taddr, uint32_t (&r)[64]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+        "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+        "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]),
+          "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]),
+          "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]),
+          "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]),
+          "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr));
+}
+
+// Statistics (and logits) of 32 accumulator columns that are already in registers: v[OFF .. OFF+31] of
+// this lane's vocabulary row.  Fewer instructions per value than drain_chunk: the column maxima come
+// from a transposed butterfly, the exponentials take one multiply-add each, and the
+// argmax ballots run only for columns whose maximum here exceeds the column's running maximum
+// (vocabulary rows are visited in ascending order, so an equal value later on never replaces the
+// index; after the first tiles a new maximum is rare).  n_cols: columns of the chunk that exist.
+template <int OFF>
+__device__ __forceinline__ void stats_chunk32(const UmmaParams& p, uint32_t (&v)[64], int lane, int row_in_tile, const TileCtx& tile,
+                                              int tok0, int n_cols, Stat& running) {
+    const int vrow = tile.v0 + row_in_tile;
+    const bool row_ok = row_in_tile < tile.rows;
+    if (p.logits != nullptr && row_ok) {
+        float* dst = p.logits + (size_t)tok0 * p.V + vrow;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            if (j < n_cols && tok0 + j < p.M) dst[(size_t)j * p.V] = __uint_as_float(v[OFF + j]);
+        }
+    }
+    const bool greedy = p.greedy != 0;
+    // column maxima by a transposed butterfly (31 exchanges for 32 columns; a warp-wide reduction
+    // instruction per column measured ten times slower): lane l ends up with the maximum of column l
+    float mine_m;
+    {
+        float zc[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float z = (row_ok && j < n_cols) ? __uint_as_float(v[OFF + j]) : -INFINITY;
+            v[OFF + j] = __float_as_uint(z);
+            zc[j] = z;
+        }
+        transposed_max(zc, lane);
+        mine_m = zc[0];
+    }
+    // Every column's maximum goes back to all lanes (it sits in lane j), which gives the lowest row attaining
+    // it and, at T > 0, the exponentials - without a branch per column (32 branches on a warp-uniform
+    // condition measured three times the cost of the whole butterfly).
+    const int warp_row0 = vrow - lane;          // vocabulary row of lane 0
+    int cand_idx = 0x7fffffff;
+    float mine_s = 0.f;
+    if (greedy) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float mxj = __shfl_sync(0xffffffffu, mine_m, j);
+            const unsigned hit = __ballot_sync(0xffffffffu, __uint_as_float(v[OFF + j]) == mxj);
+            cand_idx = lane == j ? warp_row0 + (__ffs(hit) - 1) : cand_idx;
+        }
+    } else {
+        float sums[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            const float mxj = __shfl_sync(0xffffffffu, mine_m, j);
+            const float z = __uint_as_float(v[OFF + j]);
+            const unsigned hit = __ballot_sync(0xffffffffu, z == mxj);
+            cand_idx = lane == j ? warp_row0 + (__ffs(hit) - 1) : cand_idx;
+            // (z - max) * scale as one multiply-add: -inf entries give 2^-inf = 0, an all -inf column is skipped below
+            sums[j] = exp2f(fmaf(z, p.scale_log2, -mxj * p.scale_log2));
+        }
+        transposed_sum<32>(sums, lane);
+        mine_s = mine_m == -INFINITY ? 0.f : sums[0];
+    }
+    const bool raise = mine_m > running.m;      // an equal maximum later on keeps the earlier (lower) index
+    const int new_idx = cand_idx;
+    if (raise) {
+        const float f = running.m == -INFINITY ? 0.f : exp2f((running.m - mine_m) * p.scale_log2);
+        running.s = greedy ? 0.f : mine_s + running.s * f;
+        running.m = mine_m;
+        running.idx = new_idx;
+    } else if (!greedy && mine_m != -INFINITY) {
+        running.s += mine_s * exp2f((mine_m - running.m) * p.scale_log2);
+    }
+}
+
+// ---- One pass over the weights for 257 .. 384 token rows (CTA pairs only).
+// The token rows are cut into two sub-tiles of n_tile <= 192 rows whose accumulators live in tensor memory
+// at the same time (columns 0.. and 192..), so every weight block crosses from L2 into shared memory once
+// and feeds two MMAs (the two-token-tile arrangement of lm_head_umma_kernel streams the weights twice and
+// is bound by that traffic).  Tensor memory has no room for a second pair of accumulators; instead the
+// twelve epilogue warps copy a finished sub-tile into registers (64 columns each) and hand its tensor
+// memory back before they start on its statistics, which then run from registers while the next tile's
+// MMAs are under way; the second sub-tile follows the same way.
+constexpr int kDuoEpilogueWarps = 12;      // three per TMEM lane quarter
+constexpr int kDuoThreads = (2 + kDuoEpilogueWarps) * 32;
+constexpr int kDuoSubCols = 192;           // tensor-memory columns reserved per sub-tile
+__global__ void __launch_bounds__(kDuoThreads, 1)
+lm_head_duo_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_constant__ CUtensorMap map_h, const UmmaParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t tmem_full_bar;
+    __shared__ __align__(8) uint64_t tmem_empty_bar[2];      // one per sub-tile's accumulator
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ float run_m[4][2 * kDuoSubCols];
+    __shared__ float run_s[4][2 * kDuoSubCols];
+    __shared__ int run_i[4][2 * kDuoSubCols];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int sub = p.n_tile;                                 // token rows per sub-tile
+    const int h_rows = sub / 2;                               // rows of a sub-tile this CTA loads per K block
+    const int h_bytes = h_rows * 128;
+    const int stage_bytes = kTileBytesW + 2 * h_bytes;
+    const int num_kb = p.K / kBlockK;
+    const uint32_t pair_rank = cluster_cta_rank();
+    const int group = blockIdx.x / 2;
+    constexpr int tile_rows = 2 * kVocabTile;
+    // This pair's tiles: tiles_per_group whole bands (fewer at the end of the vocabulary), then, where the bands
+    // do not divide evenly, one sub-tile of a left-over band (the pair g ^ 1 takes the other sub-tile).
+    const int n_full = max(0, min(p.tiles_per_group, p.n_bands - group * p.tiles_per_group));
+    const int n_tiles = n_full + (group < 2 * p.split_rem ? 1 : 0);
+    auto band_of = [&](int t) { return t < n_full ? group * p.tiles_per_group + t : (int)(gridDim.x / 2) * p.tiles_per_group + group / 2; };
+    auto subs_of = [&](int t) { return t < n_full ? 3 : 1 << (group & 1); };      // bit q: sub-tile q is computed
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&tmem_full_bar, 1);
+        for (int q = 0; q < 2; ++q) mbar_init(&tmem_empty_bar[q], 2 * kDuoEpilogueWarps);     // the leader's collect both CTAs' epilogue warps
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();      // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    volatile int* abort_ptr = &abort_flag;
+    pdl_wait();
+    pdl_trigger();
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint64_t pol_stream, pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            int s = 0;
+            uint32_t ph = 0;
+            uint8_t* w_dst = smem;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int v0 = band_of(t) * tile_rows + (int)pair_rank * kVocabTile;
+                const int subs = subs_of(t);
+                // both CTAs' copies complete on the leader's barrier
+                const uint32_t tx_pair = (uint32_t)(2 * (kTileBytesW + (subs == 3 ? 2 : 1) * h_bytes));
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_ptr)) { ok = false; break; }
+                    const uint32_t bar = cluster_addr(&full_bar[s], 0);
+                    if (pair_rank == 0) mbar_expect_tx_at(bar, tx_pair);
+                    tma_load_2d_pair(w_dst, &map_w128, kb * kBlockK, v0, bar, pol_stream);
+                    // rows past the end of the matrix are filled with zeros and still counted
+                    if (subs & 1) tma_load_2d_pair(w_dst + kTileBytesW, &map_h, kb * kBlockK, (int)pair_rank * h_rows, bar, pol_keep);
+                    if (subs & 2) tma_load_2d_pair(w_dst + kTileBytesW + h_bytes, &map_h, kb * kBlockK, sub + (int)pair_rank * h_rows, bar, pol_keep);
+                    w_dst += stage_bytes;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; w_dst = smem; }
+                }
+            }
+            if (!ok) {
+                for (int i = 0; i < 64; ++i) __nanosleep(2000);       // let copies in flight land
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (the pair's leader)
+        if (lane == 0 && pair_rank == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(sub >> 3) << 17) | ((uint32_t)((2 * kVocabTile) >> 4) << 24);
+            const uint32_t lo_step = (uint32_t)stage_bytes >> 4, h_step = (uint32_t)h_bytes >> 4;
+            const uint32_t a_lo0 = umma_desc_lo(smem_u32(smem));
+            int s = 0;
+            uint32_t ph = 0, a_lo = a_lo0;
+            bool ok = true;
+            for (int t = 0; t < n_tiles && ok; ++t) {
+                const int subs = subs_of(t);
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
+                    if (!mbar_wait(&full_bar[s], ph, abort_ptr)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        if (kb == 0) {       // the previous tile's accumulator has been copied out of tensor memory
+                            if (!mbar_wait(&tmem_empty_bar[q], ((uint32_t)t & 1u) ^ 1u, abort_ptr)) { ok = false; break; }
+                            tc_fence_after();
+                        }
+                        if (!((subs >> q) & 1)) continue;
+                        const uint32_t d_tmem = tmem_base + (uint32_t)(q * kDuoSubCols);
+                        const uint32_t b_lo = a_lo + (kTileBytesW >> 4) + (uint32_t)q * h_step;
+                        if (kb == 0) umma_bf16_pair<false>(d_tmem, a_lo, b_lo, idesc);
+                        else umma_bf16_pair<true>(d_tmem, a_lo, b_lo, idesc);
+                        umma_bf16_pair<true>(d_tmem, a_lo + 2, b_lo + 2, idesc);
+                        umma_bf16_pair<true>(d_tmem, a_lo + 4, b_lo + 4, idesc);
+                        umma_bf16_pair<true>(d_tmem, a_lo + 6, b_lo + 6, idesc);
+                    }
+                    if (!ok) break;
+                    umma_commit_pair(&empty_bar[s]);     // frees the stage in both CTAs
+                    a_lo += lo_step;
+                    if (++s == p.stages) { s = 0; ph ^= 1u; a_lo = a_lo0; }
+                }
+                if (ok) umma_commit_pair(&tmem_full_bar);
+            }
+        }
+    } else {
+        // ------------------------------------------------ epilogue (warps 2..13)
+        // TMEM lanes 32*quarter .. +31 are the only ones warp (quarter = warp % 4) may read; the three warps
+        // of a quarter take columns 64*part .. 64*part+63 of both sub-tiles.
+        const int quarter = warp & 3;
+        const int part = (warp - 2) >> 2;
+        const int row_in_tile = quarter * 32 + lane;
+        const int c0 = part * 64;                              // first column (token row within the sub-tile)
+        for (int c = threadIdx.x - 64; c < 4 * 2 * kDuoSubCols; c += kDuoEpilogueWarps * 32) {
+            (&run_m[0][0])[c] = -INFINITY; (&run_s[0][0])[c] = 0.f; (&run_i[0][0])[c] = 0x7fffffff;
+        }
+        asm volatile("bar.sync 1, %0;" ::"r"(kDuoEpilogueWarps * 32) : "memory");     // epilogue warps only
+        bool ok = true;
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            if (!mbar_wait_warp(&tmem_full_bar, (uint32_t)t & 1u, abort_ptr)) { ok = false; break; }
+            tc_fence_after();
+            TileCtx tile;
+            tile.v0 = band_of(t) * tile_rows + (int)pair_rank * kVocabTile;        // this CTA's 128 rows
+            tile.rows = max(0, min(kVocabTile, p.V - tile.v0));
+            const int subs = subs_of(t);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0;
+#pragma unroll 1
+            for (int q = 0; q < 2; ++q) {
+                // the sub-tile's 64 columns of this warp: into registers, and tensor memory is free for the next tile
+                uint32_t v[64];
+                const bool live = (subs >> q) & 1;             // a half-tile computes one sub-tile only
+                if (live) {
+                    tmem_load64(taddr + q * kDuoSubCols, v);
+                    tmem_wait_ld<64>(v);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_at(cluster_addr(&tmem_empty_bar[q], 0));
+                if (!live) continue;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int cc = c0 + h * 32;                // first column of the chunk within the sub-tile
+                    const int n_cols = min(32, sub - cc);
+                    if (n_cols > 0) {                           // the same in every lane
+                        const int col = q * kDuoSubCols + cc + lane;
+                        Stat running{run_m[quarter][col], run_s[quarter][col], run_i[quarter][col]};
+                        if (h == 0) stats_chunk32<0>(p, v, lane, row_in_tile, tile, q * sub + cc, n_cols, running);
+                        else stats_chunk32<32>(p, v, lane, row_in_tile, tile, q * sub + cc, n_cols, running);
+                        run_m[quarter][col] = running.m; run_s[quarter][col] = running.s; run_i[quarter][col] = running.idx;
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    // the CTA's statistics: merge the four lane quarters (ascending rows) into one partial slot
+    for (int i = threadIdx.x; i < 2 * sub; i += kDuoThreads) {
+        const int c = (i / sub) * kDuoSubCols + i % sub, tok = i;
+        if (tok < p.M) {
+            Stat acc{run_m[0][c], run_s[0][c], run_i[0][c]};
+#pragma unroll
+            for (int qd = 1; qd < 4; ++qd)
+                acc = stat_combine(acc, Stat{run_m[qd][c], run_s[qd][c], run_i[qd][c]}, p.scale_log2, p.greedy != 0);
+            const size_t slot = (size_t)(group * 2 + (int)pair_rank) * p.M;
+            p.part_max[slot + tok] = acc.m;
+            p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
+            p.part_idx[slot + tok] = acc.idx == 0x7fffffff ? acc.idx : acc.idx + p.idx_offset;
+        }
+    }
+    cluster_sync_all();      // neither CTA frees TMEM or leaves while the other may still use it
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols) : "memory");
+    }
+    if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
+}
+
 // ------------------------------------------------------------------ host side
 int sm_count() {
     static int n = 0;
@@ -508,14 +827,63 @@ int lm_head_num_partials(int M, int V) {
     return slots < kMaxCtas ? slots : kMaxCtas;
 }
 
+// 257 .. 384 token rows: two sub-tiles, one pass over the weights (lm_head_duo_kernel).
+static cudaError_t launch_lm_head_duo(const LmHeadParams& q, UmmaParams p, int ctas, cudaStream_t stream, int* n_part_used) {
+    p.n_token_tiles = 1;
+    p.n_tile = ((q.M + 1) / 2 + 15) / 16 * 16;        // rows per sub-tile, <= 192
+    const int bands = (q.V + 2 * kVocabTile - 1) / (2 * kVocabTile);
+    int groups = ctas / 2;
+    if (groups > bands) groups = bands;
+    // Whole bands per pair; a few left-over bands are cut into their two sub-tiles and dealt to the first pairs
+    // (594 bands on 74 pairs: 8 each, and 4 pairs take half a band more - not 9 each on 66 pairs).
+    p.n_bands = bands;
+    p.tiles_per_group = bands / groups;
+    p.split_rem = bands - p.tiles_per_group * groups;
+    if (2 * p.split_rem > groups) {
+        p.tiles_per_group = (bands + groups - 1) / groups;
+        groups = (bands + p.tiles_per_group - 1) / p.tiles_per_group;
+        p.split_rem = 0;
+    }
+    p.n_groups = groups;
+    const int h_rows = p.n_tile / 2;
+    const int stage_bytes = kTileBytesW + 2 * h_rows * 128;
+    int stages = kRingBytes / stage_bytes;
+    if (stages > kMaxStages) stages = kMaxStages;
+    p.stages = stages;
+    p.tmem_cols = 512;                                 // two accumulators at columns 0 and 192
+    const int slots = groups * 2;
+    if (slots > q.n_part) return cudaErrorInvalidValue;
+    *n_part_used = slots;
+    CUtensorMap map_w, map_h;
+    if (!make_tensor_map_bf16_2d(&map_w, q.lm_head, q.V, q.K, kVocabTile)) return cudaErrorInvalidValue;
+    if (!make_tensor_map_bf16_2d(&map_h, q.hidden, q.M, q.K, h_rows)) return cudaErrorInvalidValue;
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    const TimingHooks& hooks = timing_hooks();
+    if (hooks.lm_head_start && cudaEventRecord(hooks.lm_head_start, stream) != cudaSuccess) return cudaGetLastError();
+    cudaError_t e = cudaFuncSetAttribute(lm_head_duo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl_cluster(lm_head_duo_kernel, dim3(groups * 2), dim3(kDuoThreads), smem, stream, 2, map_w, map_h, p);
+    if (e != cudaSuccess) return e;
+    if (hooks.lm_head_stop && cudaEventRecord(hooks.lm_head_stop, stream) != cudaSuccess) return cudaGetLastError();
+    count_launches(1);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_part_used) {
     UmmaParams p;
     p.M = q.M; p.K = q.K; p.V = q.V;
+    int ctas = sm_count();
+    if (ctas > kMaxCtas) ctas = kMaxCtas;
+    p.greedy = q.greedy;
+    p.scale_log2 = q.inv_T_log2e;
+    p.logits = q.logits;
+    p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
+    p.dev_status = q.dev_status;
+    p.idx_offset = q.idx_offset;
+    if (q.M > 256 && q.M <= 2 * kDuoSubCols) return launch_lm_head_duo(q, p, ctas, stream, n_part_used);
     p.n_token_tiles = q.M > 256 ? 2 : 1;
     const int per_tile = (q.M + p.n_token_tiles - 1) / p.n_token_tiles;
     p.n_tile = (per_tile + 15) / 16 * 16;
-    int ctas = sm_count();
-    if (ctas > kMaxCtas) ctas = kMaxCtas;
     // From 64 token rows up, pairs of CTAs (cta_group::2) share the hidden-state tile: the traffic
     // from L2 into shared memory per weight byte drops from 1 + N/128 to 1 + N/256.
     const bool pair = p.n_tile >= kPairMinTile;

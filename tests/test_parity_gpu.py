@@ -228,6 +228,15 @@ ODD_SHAPES = [
          temperature=0.0, ctx_lo=60, ctx_hi=260),
     dict(name="one_tile_d64", batch=5, gamma=1, n_q_heads=6, n_kv_heads=3, head_dim=64, hidden=128, vocab=512,
          temperature=1.3, ctx_lo=0, ctx_hi=500),
+    # 257 .. 384 LM-head rows (the one-pass, three-sub-tile arrangement): sub-tiles of 112 rows (a 16-column
+    # tail) and of 96 rows, a ragged last vocabulary band, both temperatures
+    dict(name="rows301_t1", batch=43, gamma=6, n_q_heads=2, n_kv_heads=1, head_dim=64, hidden=320, vocab=3000,
+         temperature=0.9, ctx_lo=0, ctx_hi=40),
+    dict(name="rows272_t0", batch=34, gamma=7, n_q_heads=2, n_kv_heads=2, head_dim=64, hidden=192, vocab=8200,
+         temperature=0.0, ctx_lo=1, ctx_hi=50),
+    # 76 vocabulary bands on 74 CTA pairs: the two left-over bands (the last one ragged) are cut into half-tiles
+    dict(name="rows384_split_bands", batch=64, gamma=5, n_q_heads=2, n_kv_heads=1, head_dim=64, hidden=128, vocab=19400,
+         temperature=1.1, ctx_lo=0, ctx_hi=30),
 ]
 
 
