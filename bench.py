@@ -394,7 +394,8 @@ def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=Non
     }
 
     if want_tvd and sampling and cfg.gamma >= 1:
-        # the paper's distribution-alignment diagnostic (Eq. 6) on the logits the step just wrote
+        # the paper's distribution-alignment diagnostic (Eq. 6) on the logits the step just wrote, with the row
+        # statistics the acceptance call left in its workspace (one read of the logits)
         ws = mv.alloc_workspace(mv.massv_tvd_workspace_size(step.cdesc), dev)
         tvd = torch.empty((cfg.batch, cfg.gamma), dtype=torch.float32, device=dev)
         acc = torch.empty_like(tvd)
@@ -403,7 +404,7 @@ def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=Non
             flush.fill_(1)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
-            mv.massv_tvd(step.cdesc, step.logits, w["draft_probs"], tvd, acc, ws, step.dev_status)
+            mv.massv_tvd_after_accept(step.cdesc, step.logits, w["draft_probs"], step.accept_ws, tvd, acc, ws, step.dev_status)
             b.record(stream)
             torch.cuda.synchronize()
             if i >= 3:

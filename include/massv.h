@@ -86,8 +86,15 @@ typedef struct massv_accept_desc {
     int32_t hidden;              /* K, a multiple of 64 */
     int32_t vocab;               /* V, a multiple of 8 */
     float temperature;           /* T >= 0; 0 selects greedy verification */
-    uint32_t flags;              /* reserved, 0 */
+    uint32_t flags;              /* reserved, 0 (see MASSV_TEST_SKIP_STAGE below) */
 } massv_accept_desc;
+
+/* Only in a library compiled with -DMASSV_TEST_HOOKS (the test suite builds one beside the product, with a
+ * short MASSV_SPIN_LIMIT): massv_accept_desc.flags = MASSV_TEST_SKIP_STAGE makes the LM-head kernel's
+ * producer withhold one pipeline stage - no bytes announced, no copy issued - so that the consumer's
+ * bounded wait runs out and the call reports MASSV_ERR_TIMEOUT in dev_status instead of waiting for ever.
+ * The product library refuses any non-zero flags. */
+#define MASSV_TEST_SKIP_STAGE 0x80000000u
 
 /* Bytes of scratch massv_verify_attn needs for this geometry (0 on a bad descriptor). */
 size_t massv_verify_attn_workspace_size(const massv_attn_desc *desc);
@@ -184,7 +191,7 @@ int massv_accept(const massv_accept_desc *desc, const void *hidden, const void *
  *
  * It computes exactly what massv_accept computes, with the same kernels and the
  * same arguments, except:
- *   - there is no workspace argument.  Scratch is a fixed array of about 640 KiB
+ *   - there is no workspace argument.  Scratch is a fixed array of about 210 KiB
  *     of device memory that belongs to the library image: every GPU that loads
  *     the library holds it until the process exits, used or not.
  *   - the fp32 logits have no room in that array, so at T > 0 logits_out is
@@ -194,9 +201,13 @@ int massv_accept(const massv_accept_desc *desc, const void *hidden, const void *
  *     returns MASSV_ERR_WORKSPACE and launches nothing.
  *   - the first call on each device looks up the array's device address (the
  *     device that is current at the call).  Make that first call during start-up,
- *     outside any stream capture.  Later calls on that device reuse the address.
+ *     outside any stream capture.  Later calls on that device reuse the address,
+ *     which is remembered per device ordinal: after a cudaDeviceReset (which
+ *     unloads the library image from the device) it is stale, so do not reset a
+ *     device between calls.
  *   - all calls on one device share the one array, and it keeps what the last
- *     call left in it.  The call clears the part that has to start at zero.  Two
+ *     call left in it (every part is rewritten by the call's own kernels before
+ *     it is read, so nothing stale is used).  Two
  *     calls that can run on the GPU at the same time (different streams without
  *     an ordering between them) would overwrite each other's scratch: keep calls
  *     on one stream or order them yourself.
@@ -228,6 +239,23 @@ size_t massv_tvd_workspace_size(const massv_accept_desc *desc);
 int massv_tvd(const massv_accept_desc *desc, const float *logits, const float *draft_probs,
               float *tvd_out, float *accept_prob_out,
               void *workspace, size_t workspace_bytes, int32_t *dev_status, massv_stream_t stream);
+
+/*
+ * The same diagnostic (Eq. 6) right after massv_accept on the same stream, with ONE read of the logits:
+ * massv_accept leaves every row's merged softmax statistics (max logit, sum of exp((z - max)/T)) in its
+ * workspace, and this call takes them from there instead of computing them again, so it reads each
+ * drafted row of the logits and of q once (B*gamma*V*8 bytes).
+ *   desc                  the descriptor massv_accept was called with (T > 0, gamma >= 1)
+ *   logits                the logits_out of that massv_accept call
+ *   accept_workspace      the workspace of that call, untouched since (its size is checked)
+ *   tvd_out, accept_prob_out, workspace (massv_tvd_workspace_size bytes): as for massv_tvd
+ * The statistics come from the LM-head kernel's fp32 arithmetic; results agree with massv_tvd's to
+ * rounding (both are held to 1e-4 absolute against a double-precision evaluation).
+ */
+int massv_tvd_after_accept(const massv_accept_desc *desc, const float *logits, const float *draft_probs,
+                           const void *accept_workspace, size_t accept_workspace_bytes,
+                           float *tvd_out, float *accept_prob_out,
+                           void *workspace, size_t workspace_bytes, int32_t *dev_status, massv_stream_t stream);
 
 /*
  * Commit or roll back the speculative block (Sec. 2.1: accepted tokens are

@@ -58,6 +58,8 @@ def _load():
     lib.massv_tvd_workspace_size.argtypes = [ctypes.POINTER(AcceptDesc)]
     lib.massv_tvd.restype = ctypes.c_int
     lib.massv_tvd.argtypes = [ctypes.POINTER(AcceptDesc), f32p, f32p, f32p, f32p, vp, ctypes.c_size_t, i32p, vp]
+    lib.massv_tvd_after_accept.restype = ctypes.c_int
+    lib.massv_tvd_after_accept.argtypes = [ctypes.POINTER(AcceptDesc), f32p, f32p, vp, ctypes.c_size_t, f32p, f32p, vp, ctypes.c_size_t, i32p, vp]
     lib.massv_tvd_histogram.restype = ctypes.c_int
     lib.massv_tvd_histogram.argtypes = [ctypes.c_int64, f32p, ctypes.c_int32, vp, vp]
     lib.massv_sample_top_p.restype = ctypes.c_int
@@ -237,6 +239,18 @@ def massv_tvd(desc, logits, draft_probs, tvd_out, accept_prob_out=None, workspac
                         _ptr(dev_status, torch.int32), _stream())
     if rc != 0:
         raise MassvError(rc, "massv_tvd")
+
+
+def massv_tvd_after_accept(desc, logits, draft_probs, accept_workspace, tvd_out, accept_prob_out=None, workspace=None,
+                           dev_status=None) -> None:
+    """massv_tvd with one read of the logits: the row statistics come from the workspace that the
+    massv_accept call with the same descriptor has just used."""
+    f32 = torch.float32
+    rc = _lib.massv_tvd_after_accept(ctypes.byref(desc), _ptr(logits, f32), _ptr(draft_probs, f32), _ptr(accept_workspace),
+                                     accept_workspace.numel(), _ptr(tvd_out, f32), _ptr(accept_prob_out, f32), _ptr(workspace),
+                                     workspace.numel() if workspace is not None else 0, _ptr(dev_status, torch.int32), _stream())
+    if rc != 0:
+        raise MassvError(rc, "massv_tvd_after_accept")
 
 
 def massv_tvd_histogram(tvd, counts) -> None:

@@ -99,7 +99,10 @@ __global__ void __launch_bounds__(kScanThreads) accept_scan_kernel(AcceptParams 
             // both partners must form the same sum: order the operands by lane
             acc = (lane & o) ? combine(y, acc, inv_T) : combine(acc, y, inv_T);
         }
-        if (lane == 0) row_stat[warp] = acc;
+        if (lane == 0) {
+            row_stat[warp] = acc;
+            if (p.row_stats) { p.row_stats[(size_t)row * 2] = acc.m; p.row_stats[(size_t)row * 2 + 1] = acc.s; }
+        }
     }
     __syncthreads();
     if (warp != 0) return;

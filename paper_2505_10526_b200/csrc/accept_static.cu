@@ -19,7 +19,7 @@ namespace {
 constexpr int kStaticMaxRows = 64;          // B * (gamma + 1)
 constexpr int kStaticMaxBatch = 64;
 constexpr int kStaticMaxVocab = 524288;
-constexpr int kStaticMaxParts = 768;        // upper bound of lm_head_num_partials()
+constexpr int kStaticMaxParts = 192;        // lm_head_num_partials() never exceeds this (one slot per CTA, at most 192 CTAs)
 constexpr int kStaticMaxChunks = kStaticMaxVocab / kResidualChunk;
 
 constexpr size_t kA = 256;
@@ -30,7 +30,7 @@ constexpr size_t kOffIdx = kOffSum + up((size_t)kStaticMaxParts * kStaticMaxRows
 constexpr size_t kOffState = kOffIdx + up((size_t)kStaticMaxParts * kStaticMaxRows * sizeof(int32_t));
 constexpr size_t kOffChunks = kOffState + up((size_t)kStaticMaxBatch * sizeof(SeqState));
 constexpr size_t kOffCounters = kOffChunks + up((size_t)kStaticMaxBatch * kStaticMaxChunks * sizeof(double));
-constexpr size_t kScratchBytes = kOffCounters + up((size_t)kStaticMaxBatch * sizeof(unsigned int));   // about 640 KiB
+constexpr size_t kScratchBytes = kOffCounters + up((size_t)kStaticMaxBatch * sizeof(unsigned int));   // about 210 KiB
 
 // The scratch itself.  In host code this name is only a handle for
 // cudaGetSymbolAddress; it is not a device address.
@@ -88,11 +88,9 @@ extern "C" int massv_accept_static(const massv_accept_desc* desc, const void* hi
     const int rc = scratch_address(&ws);
     if (rc != MASSV_OK) return rc;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    // The array keeps whatever the previous call left.  The arrival counters are
-    // the only part that must start at zero; everything else is written before
-    // it is read.
-    if (cudaMemsetAsync(ws + kOffCounters, 0, (size_t)desc->batch * sizeof(unsigned int), s) != cudaSuccess)
-        return MASSV_ERR_CUDA;
+    // The array keeps whatever the previous call left.  Nothing in it has to be cleared from the host:
+    // every part is written by a kernel of this call before a later kernel reads it (the arrival
+    // counters of the residual draw are zeroed by the scan kernel that runs before it).
 
     LmHeadParams g;
     g.M = (int)M; g.K = desc->hidden; g.V = desc->vocab;

@@ -51,6 +51,11 @@ int check_attn_desc(const massv_attn_desc* d) {
     if ((d->n_q_heads / d->n_kv_heads) * (d->gamma + 1) > 64) return MASSV_ERR_UNSUPPORTED;
     if (d->kv_chunk % 64 != 0 || d->kv_chunk > 4096) return MASSV_ERR_UNSUPPORTED;
     if (d->flags > MASSV_ATTN_KERNEL_TCGEN05) return MASSV_ERR_UNSUPPORTED;
+    {
+        // the chunk merge kernel indexes at most 1024 chunks per sequence: refuse here, before anything is launched
+        const long chunk = d->kv_chunk > 0 ? d->kv_chunk : auto_kv_chunk(*d);
+        if (((long)d->max_pages_per_seq * kPageSize + chunk - 1) / chunk > 1024) return MASSV_ERR_UNSUPPORTED;
+    }
     return MASSV_OK;
 }
 
@@ -83,13 +88,17 @@ int check_accept_desc(const massv_accept_desc* d) {
     if (d->gamma > kMaxRows - 1) return MASSV_ERR_UNSUPPORTED;
     if ((long)d->batch * (d->gamma + 1) > 512) return MASSV_ERR_UNSUPPORTED;
     if (d->hidden % 64 != 0 || d->vocab % 8 != 0) return MASSV_ERR_UNSUPPORTED;
+#ifdef MASSV_TEST_HOOKS
+    if ((d->flags & ~MASSV_TEST_SKIP_STAGE) != 0) return MASSV_ERR_UNSUPPORTED;
+#else
     if (d->flags != 0) return MASSV_ERR_UNSUPPORTED;
+#endif
     return MASSV_OK;
 }
 
 struct AcceptLayout {
     int n_part, n_chunks;
-    size_t off_max, off_sum, off_idx, off_state, off_chunks, off_counters, off_logits, total;
+    size_t off_max, off_sum, off_idx, off_state, off_chunks, off_counters, off_rowstat, off_logits, total;
 };
 
 AcceptLayout accept_layout(const massv_accept_desc& d) {
@@ -104,6 +113,7 @@ AcceptLayout accept_layout(const massv_accept_desc& d) {
     l.off_state = off; off += align_up((size_t)d.batch * sizeof(SeqState), kAlign);
     l.off_chunks = off; off += align_up((size_t)d.batch * l.n_chunks * sizeof(double), kAlign);
     l.off_counters = off; off += align_up((size_t)d.batch * sizeof(unsigned int), kAlign);
+    l.off_rowstat = off; off += align_up(M * 2 * sizeof(float), kAlign);
     l.off_logits = off;
     if (d.temperature > 0.f) off += align_up(M * (size_t)d.vocab * sizeof(float), kAlign);
     l.total = off;
@@ -195,6 +205,9 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
     g.part_sum = reinterpret_cast<float*>(ws + l.off_sum);
     g.part_idx = reinterpret_cast<int32_t*>(ws + l.off_idx);
     g.dev_status = dev_status;
+#ifdef MASSV_TEST_HOOKS
+    g.test_skip_stage = (desc->flags & MASSV_TEST_SKIP_STAGE) ? 1 : 0;
+#endif
     int n_part_used = 0;
     if (launch_lm_head(g, s, &n_part_used) != cudaSuccess) return MASSV_ERR_CUDA;
 
@@ -207,6 +220,7 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
     a.seq_state = reinterpret_cast<SeqState*>(ws + l.off_state);
     a.chunk_sums = reinterpret_cast<double*>(ws + l.off_chunks);
     a.counters = reinterpret_cast<unsigned int*>(ws + l.off_counters);
+    a.row_stats = reinterpret_cast<float*>(ws + l.off_rowstat);
     a.n_chunks = l.n_chunks;
     a.dev_status = dev_status;
     return launch_accept(a, s) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
@@ -392,13 +406,13 @@ size_t massv_tvd_workspace_size(const massv_accept_desc* desc) {
     return align_up(rows * kTvdSlices * sizeof(float), kAlign) + 3 * align_up(rows * kTvdSlices * sizeof(double), kAlign);
 }
 
-int massv_tvd(const massv_accept_desc* desc, const float* logits, const float* draft_probs, float* tvd_out,
-              float* accept_prob_out, void* workspace, size_t workspace_bytes, int32_t* dev_status, massv_stream_t stream) {
-    (void)dev_status;
+static int tvd_call(const massv_accept_desc* desc, const float* logits, const float* draft_probs, const float* row_stats, float* tvd_out,
+                    float* accept_prob_out, void* workspace, size_t workspace_bytes, massv_stream_t stream) {
     const int rc = check_accept_desc(desc);
     if (rc != MASSV_OK) return rc;
     if (desc->gamma < 1 || !(desc->temperature > 0.f)) return MASSV_ERR_INVALID_ARG;
     if (!logits || !draft_probs || !tvd_out) return MASSV_ERR_INVALID_ARG;
+    if (!aligned16(logits) || !aligned16(draft_probs)) return MASSV_ERR_INVALID_ARG;
     const size_t need = massv_tvd_workspace_size(desc);
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0 || workspace_bytes < need) return MASSV_ERR_WORKSPACE;
     const size_t rows = (size_t)desc->batch * desc->gamma;
@@ -412,7 +426,27 @@ int massv_tvd(const massv_accept_desc* desc, const float* logits, const float* d
     t.slice_sum = reinterpret_cast<double*>(ws + off);
     t.slice_abs = reinterpret_cast<double*>(ws + off + step);
     t.slice_min = reinterpret_cast<double*>(ws + off + 2 * step);
+    t.row_stats = row_stats;
     return launch_tvd(t, reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? MASSV_OK : MASSV_ERR_CUDA;
+}
+
+int massv_tvd(const massv_accept_desc* desc, const float* logits, const float* draft_probs, float* tvd_out,
+              float* accept_prob_out, void* workspace, size_t workspace_bytes, int32_t* dev_status, massv_stream_t stream) {
+    (void)dev_status;
+    return tvd_call(desc, logits, draft_probs, nullptr, tvd_out, accept_prob_out, workspace, workspace_bytes, stream);
+}
+
+int massv_tvd_after_accept(const massv_accept_desc* desc, const float* logits, const float* draft_probs,
+                           const void* accept_workspace, size_t accept_workspace_bytes, float* tvd_out, float* accept_prob_out,
+                           void* workspace, size_t workspace_bytes, int32_t* dev_status, massv_stream_t stream) {
+    (void)dev_status;
+    const int rc = check_accept_desc(desc);
+    if (rc != MASSV_OK) return rc;
+    const AcceptLayout l = accept_layout(*desc);
+    if (!accept_workspace || (reinterpret_cast<uintptr_t>(accept_workspace) % kAlign) != 0 || accept_workspace_bytes < l.total)
+        return MASSV_ERR_WORKSPACE;
+    const float* row_stats = reinterpret_cast<const float*>(static_cast<const char*>(accept_workspace) + l.off_rowstat);
+    return tvd_call(desc, logits, draft_probs, row_stats, tvd_out, accept_prob_out, workspace, workspace_bytes, stream);
 }
 
 int massv_tvd_histogram(int64_t n, const float* tvd, int32_t bins, int64_t* counts, massv_stream_t stream) {
@@ -457,7 +491,7 @@ const char* massv_strerror(int status) {
     }
 }
 
-int massv_version(void) { return 100; }
+int massv_version(void) { return 101; }
 
 int massv_set_timing_events(massv_event_t lm_head_start, massv_event_t lm_head_stop, massv_event_t attn_start,
                             massv_event_t attn_stop) {

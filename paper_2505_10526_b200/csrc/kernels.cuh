@@ -56,6 +56,7 @@ struct LmHeadParams {
     int32_t* part_idx;              // [n_part, M]
     int32_t* dev_status;
     int idx_offset = 0;             // added to the argmax indices (first vocabulary row of a shard)
+    int test_skip_stage = 0;        // test builds only: the producer withholds one stage (see MASSV_TEST_SKIP_STAGE)
 };
 int lm_head_num_partials(int M, int V);            // upper bound of the partial slots, for workspace sizing
 // *n_part_used receives the number of slots this launch fills (<= p.n_part).
@@ -74,6 +75,7 @@ struct AcceptParams {
     int32_t *out_tokens, *accept_len;
     float* probs_out;               // optional
     SeqState* seq_state;            // [B]
+    float* row_stats = nullptr;     // optional [B*(gamma+1), 2]: the merged (max logit, sum exp((z - max)/T)) of every row
     double* chunk_sums;             // [B, n_chunks]
     unsigned int* counters;         // [B]
     int n_chunks;
@@ -141,6 +143,7 @@ struct TvdParams {
     float *tvd_out, *accept_prob_out;
     float* slice_max;               // [B*gamma, kTvdSlices]
     double *slice_sum, *slice_abs, *slice_min;
+    const float* row_stats = nullptr;   // [B*(gamma+1), 2] left by the acceptance scan: then the statistics pass is skipped
 };
 cudaError_t launch_tvd(const TvdParams& p, cudaStream_t stream);
 

@@ -51,6 +51,7 @@ struct UmmaParams {
     int32_t* part_idx;
     int32_t* dev_status;
     int idx_offset;      // added to the argmax indices that leave the kernel
+    int test_skip_stage = 0;   // test builds only: withhold the second K block of the first tile
     int n_bands = 0;     // duo kernel: 256-row vocabulary bands in all
     int split_rem = 0;   // duo kernel: bands left over after tiles_per_group per pair, each cut in two half-tiles (one sub-tile each)
 };
@@ -356,6 +357,15 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
                 const uint32_t tx_bytes = (uint32_t)(rows * 128 + p.n_tile * 128);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_ptr)) { ok = false; break; }
+#ifdef MASSV_TEST_HOOKS
+                    if (p.test_skip_stage && t == 0 && kb == 1) {
+                        // nothing is announced and nothing is copied for this stage: the MMA thread's wait for it
+                        // must give up by itself
+                        w_dst += stage_bytes;
+                        if (++s == p.stages) { s = 0; ph ^= 1u; w_dst = smem; }
+                        continue;
+                    }
+#endif
                     uint8_t* h_dst = w_dst + kTileBytesW;
                     if constexpr (PAIR) {
                         // Both CTAs' copies complete on the leader's barrier; the leader announces the
@@ -880,6 +890,7 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
     p.dev_status = q.dev_status;
     p.idx_offset = q.idx_offset;
+    p.test_skip_stage = q.test_skip_stage;
     if (q.M > 256 && q.M <= 2 * kDuoSubCols) return launch_lm_head_duo(q, p, ctas, stream, n_part_used);
     p.n_token_tiles = q.M > 256 ? 2 : 1;
     const int per_tile = (q.M + p.n_token_tiles - 1) / p.n_token_tiles;

@@ -6,7 +6,10 @@
 
 namespace massv {
 
-constexpr uint32_t kSpinLimit = 1u << 24;   // polls before a device-side wait gives up
+#ifndef MASSV_SPIN_LIMIT
+#define MASSV_SPIN_LIMIT (1u << 24)
+#endif
+constexpr uint32_t kSpinLimit = MASSV_SPIN_LIMIT;   // polls before a device-side wait gives up (a test build shortens it)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

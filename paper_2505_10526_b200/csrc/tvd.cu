@@ -3,7 +3,8 @@
 //     TVD(p_j, q_j) = 1/2 * sum_v |p_j(v) - q_j(v)|,      p_j = softmax(z_j / T)
 // and the acceptance probability of the rejection test, sum_v min(p_j(v), q_j(v)) = 1 - TVD.
 // Three small kernels over fixed vocabulary slices, every reduction in a fixed order:
-//   tvd_stats_kernel   per (row, slice): max logit and sum of exponentials;
+//   tvd_stats_kernel   per (row, slice): max logit and sum of exponentials (skipped when the caller hands in
+//                      the statistics the acceptance call left behind: then the logits are read once);
 //   tvd_sum_kernel     per (row, slice): merge the row's slice statistics, then sum |p-q| and min(p,q);
 //   tvd_final_kernel   per row: add the slices in order.
 #include "kernels.cuh"
@@ -80,11 +81,19 @@ __global__ void __launch_bounds__(kThreadsTvd) tvd_sum_kernel(TvdParams p) {
     pdl_trigger();
     const int slice = blockIdx.x, row = blockIdx.y;
     float M = -INFINITY;
-    for (int s = 0; s < kTvdSlices; ++s) M = fmaxf(M, p.slice_max[row * kTvdSlices + s]);
     double S = 0.0;
-    for (int s = 0; s < kTvdSlices; ++s) {
-        const float ms = p.slice_max[row * kTvdSlices + s];
-        if (ms > -INFINITY) S += p.slice_sum[row * kTvdSlices + s] * (double)expf((ms - M) * p.inv_T);
+    if (p.row_stats) {
+        // the acceptance scan's merged statistics of logits row b*(gamma+1)+j
+        const int b = row / p.gamma, j = row % p.gamma;
+        const float2 ms = *reinterpret_cast<const float2*>(p.row_stats + (size_t)(b * (p.gamma + 1) + j) * 2);
+        M = ms.x;
+        S = (double)ms.y;
+    } else {
+        for (int s = 0; s < kTvdSlices; ++s) M = fmaxf(M, p.slice_max[row * kTvdSlices + s]);
+        for (int s = 0; s < kTvdSlices; ++s) {
+            const float ms = p.slice_max[row * kTvdSlices + s];
+            if (ms > -INFINITY) S += p.slice_sum[row * kTvdSlices + s] * (double)expf((ms - M) * p.inv_T);
+        }
     }
     const float inv_sum = (float)(1.0 / S);
     const int v0 = slice * p.slice_len, v1 = min(p.V, v0 + p.slice_len);
@@ -129,13 +138,17 @@ __global__ void tvd_final_kernel(TvdParams p) {
 
 cudaError_t launch_tvd(const TvdParams& p, cudaStream_t stream) {
     const int rows = p.B * p.gamma;
-    cudaError_t e = launch_pdl(tvd_stats_kernel, dim3(kTvdSlices, rows), dim3(kThreadsTvd), 0, stream, p);
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (!p.row_stats) {
+        e = launch_pdl(tvd_stats_kernel, dim3(kTvdSlices, rows), dim3(kThreadsTvd), 0, stream, p);
+        if (e != cudaSuccess) return e;
+        count_launches(1);
+    }
     e = launch_pdl(tvd_sum_kernel, dim3(kTvdSlices, rows), dim3(kThreadsTvd), 0, stream, p);
     if (e != cudaSuccess) return e;
     e = launch_pdl(tvd_final_kernel, dim3((rows + 127) / 128), dim3(128), 0, stream, p);
     if (e != cudaSuccess) return e;
-    count_launches(3);
+    count_launches(2);
     return cudaGetLastError();
 }
 

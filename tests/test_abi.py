@@ -100,3 +100,15 @@ def test_timing_hook_rejects_half_a_pair(mv):
     assert lib.massv_set_timing_events(ctypes.c_void_p(8), None, None, None) == -1
     assert lib.massv_set_timing_events(None, None, None, ctypes.c_void_p(8)) == -1
     assert lib.massv_set_timing_events(None, None, None, None) == 0
+
+
+def test_attention_refuses_more_chunks_than_the_merge_can_index(mv):
+    """A forced 64-token chunk on a page table of more than 65,536 tokens per sequence would need more than
+    1024 chunks: refused on the host (size query 0, call -2), nothing launched."""
+    d = mv.attn_desc(1, 5, 4, 1, 64, 4097, 5000, kv_chunk=64)          # 65,552 tokens per sequence
+    assert mv.massv_verify_attn_workspace_size(d) == 0
+    lib = mv.binding._lib
+    fake = 0x1000
+    assert lib.massv_verify_attn(ctypes.byref(d), fake, fake, fake, fake, fake, fake, fake, fake, None, None, fake, 1 << 30, None, None) == -2
+    ok = mv.attn_desc(1, 5, 4, 1, 64, 4096, 5000, kv_chunk=64)         # exactly 1024 chunks
+    assert mv.massv_verify_attn_workspace_size(ok) > 0

@@ -328,11 +328,14 @@ def test_sliding_window_attention(name, window, kv_chunk, subset):
     run_case(name, subset=subset, check_determinism=False, window=window, kv_chunk=kv_chunk)
 
 
+@pytest.mark.parametrize("fused", [False, True], ids=["own_statistics", "after_accept"])
 @pytest.mark.parametrize("name,subset", [("tiny_ragged_t1", None), ("tiny_peaked_t1", None), ("qwen7b_b16_t1", [0, 5, 15])])
-def test_tvd_diagnostic_matches_oracle(name, subset):
+def test_tvd_diagnostic_matches_oracle(name, subset, fused):
     """massv_tvd (Eq. 6) against the oracle's TVD of (softmax of oracle logits, q), row by row;
     1 - TVD must equal the acceptance probability output.  Tolerance 1e-4 absolute, the
-    tolerance of the probabilities it is a sum of differences of."""
+    tolerance of the probabilities it is a sum of differences of.  Both forms: the stand-alone call
+    that computes the rows' softmax statistics itself, and massv_tvd_after_accept, which takes them
+    from the acceptance call's workspace and reads the logits once."""
     import paper_2505_10526_b200 as mv
     cfg = get_config(name)
     w = generate(cfg, device="cuda", with_attention=False)
@@ -345,7 +348,10 @@ def test_tvd_diagnostic_matches_oracle(name, subset):
                     toks, lens, logits, None, ws, None)
     tvd = torch.zeros((B, g), dtype=torch.float32, device="cuda"); acc = torch.zeros_like(tvd)
     ws2 = mv.alloc_workspace(mv.massv_tvd_workspace_size(desc), "cuda")
-    mv.massv_tvd(desc, logits, w["draft_probs"], tvd, acc, ws2, None)
+    if fused:
+        mv.massv_tvd_after_accept(desc, logits, w["draft_probs"], ws, tvd, acc, ws2, None)
+    else:
+        mv.massv_tvd(desc, logits, w["draft_probs"], tvd, acc, ws2, None)
     torch.cuda.synchronize()
     idx = list(range(B)) if subset is None else subset
     hid = oracle.bf16_bits(w["hidden"])[idx].reshape(len(idx) * R, cfg.hidden)
