@@ -48,11 +48,11 @@ MIN_SPLIT_STEPS = 5
 # device) and scaled by the K/V bytes of the launch: the kernel streams every K/V byte once, so its
 # traffic grows in proportion.  None: no capture of the kernel as it stands.
 NCU_TRAFFIC_RATIO = {
-    ("attn", "qwen"): None,
-    ("attn", "gemma"): None,
-    ("lm_head", "qwen"): None,
+    ("attn", "qwen"): 693.4 / 691.5,          # profiles/attn_umma_kernel_qwen7b_long_b16.md (batch 16, scaled by K/V bytes)
+    ("attn", "gemma"): 1.384 / 1.34,          # profiles/attn_split_kernel_gemma12b_b32_t1.md (read 1.378 GB + 6.2 MB written)
+    ("lm_head", "qwen"): 1.0934 / 1.0900,     # profiles/lm_head_umma_kernel_qwen7b_b1_t0.md (the weight-bound launches, M <= 256)
     ("lm_head", "gemma"): None,
-    ("residual", "qwen"): None,
+    ("residual", "qwen"): (74.39 + 1.85) / 77.86,   # profiles/residual_sample_kernel_qwen7b_lmhead_g5_t1.md
     ("residual", "gemma"): None,
 }
 
