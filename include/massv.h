@@ -101,7 +101,7 @@ size_t massv_verify_attn_workspace_size(const massv_attn_desc *desc);
 
 /*
  * Target attention for the block rows (Sec. 2.1: the target scores positions
- * t+1 .. t+gamma+1 "in parallel with one forward call"; Sec. 2.2: the context
+ * t+1 .. t+gamma+1 of a drafted block in a single pass; Sec. 2.2: the context
  * is m projected image features followed by text tokens).
  *
  * For sequence b with committed length L_b = seq_lens[b]:

@@ -96,6 +96,9 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint32_t a_lo, u
         : "memory");
 }
 // Arrive, in both CTAs of the pair, on the barrier at this shared-memory offset once the MMAs issued so far are done.
+// This barrier arrive between the two CTAs of one pair (same GPU) is the only multicast qualifier in the sources:
+// every TMA load here (tma_load_2d, tma_load_2d_pair, the 1-D bulk copies) is non-multicast and reads this GPU's
+// memory only.
 __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
                  "h"((uint16_t)3)
@@ -191,25 +194,6 @@ __device__ __forceinline__ void transposed_sum(float (&v)[C], int lane) {
         } else {
             v[0] += __shfl_xor_sync(0xffffffffu, v[0], offset);
         }
-    }
-}
-
-// The same exchange pattern for maxima: on return lane l holds the maximum of column l over the 32 lanes.
-__device__ __forceinline__ void transposed_max(float (&v)[32], int lane) {
-    int n = 32;
-#pragma unroll
-    for (int offset = 16; offset >= 1; offset >>= 1) {
-        const int half = n / 2;
-        const bool upper = (lane & offset) != 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            if (i < half) {
-                const float send = upper ? v[i] : v[i + half];
-                const float keep = upper ? v[i + half] : v[i];
-                v[i] = fmaxf(keep, __shfl_xor_sync(0xffffffffu, send, offset));
-            }
-        }
-        n = half;
     }
 }
 
@@ -520,94 +504,160 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
     if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
 }
 
-// 64 accumulator columns of this thread's lane (vocabulary row) in one load.
-__device__ __forceinline__ void tmem_load64(uint32_t taddr, uint32_t (&r)[64]) {
+// 16 TMEM lanes x 64 columns -> 32 registers per thread.  Register 4k+e holds row (lane/4 + 8*(e>>1)) of the
+// 16, column 8k + 2*(lane%4) + (e&1) of the 64.  (No wait: the caller waits once for all its loads.)
+__device__ __forceinline__ void tmem_load_16x64(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+        "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
-        "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
-        "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]),
-          "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]),
-          "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]),
-          "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]),
-          "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
 }
 
-// Statistics (and logits) of 32 accumulator columns that are already in registers: v[OFF .. OFF+31] of
-// this lane's vocabulary row.  Fewer instructions per value than drain_chunk: the column maxima come
-// from a transposed butterfly, the exponentials take one multiply-add each, and the
-// argmax ballots run only for columns whose maximum here exceeds the column's running maximum
-// (vocabulary rows are visited in ascending order, so an equal value later on never replaces the
-// index; after the first tiles a new maximum is rare).  n_cols: columns of the chunk that exist.
-template <int OFF>
-__device__ __forceinline__ void stats_chunk32(const UmmaParams& p, uint32_t (&v)[64], int lane, int row_in_tile, const TileCtx& tile,
-                                              int tok0, int n_cols, Stat& running) {
-    const int vrow = tile.v0 + row_in_tile;
-    const bool row_ok = row_in_tile < tile.rows;
-    if (p.logits != nullptr && row_ok) {
-        float* dst = p.logits + (size_t)tok0 * p.V + vrow;
+// Reduction of 16 per-thread values (one per column the thread sees) over the eight lanes that hold the same
+// columns for other rows (lanes that differ in lane / 4): a transposed butterfly of 8 + 4 + 2 exchanges, after
+// which a[0], a[1] belong to columns 2 * (lane / 4) and 2 * (lane / 4) + 1 of the thread's 16.
+struct OpMax { __device__ __forceinline__ float operator()(float x, float y) const { return fmaxf(x, y); } };
+struct OpAdd { __device__ __forceinline__ float operator()(float x, float y) const { return x + y; } };
+struct OpMin { __device__ __forceinline__ float operator()(float x, float y) const { return fminf(x, y); } };
+template <typename Op>
+__device__ __forceinline__ void reduce_over_row_lanes(float (&a)[16], int lane, Op op) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            if (j < n_cols && tok0 + j < p.M) dst[(size_t)j * p.V] = __uint_as_float(v[OFF + j]);
+    for (int half = 8; half >= 2; half >>= 1) {
+        const int offset = 2 * half;                      // 16, 8, 4
+        const bool upper = (lane & offset) != 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (i < half) {
+                const float send = upper ? a[i] : a[i + half];
+                const float keep = upper ? a[i + half] : a[i];
+                a[i] = op(keep, __shfl_xor_sync(0xffffffffu, send, offset));
+            }
         }
     }
+}
+// The reverse: a[0], a[1] of every lane go back to all eight lanes, in column order (2 + 4 + 8 exchanges).
+__device__ __forceinline__ void gather_over_row_lanes(float (&a)[16], int lane) {
+#pragma unroll
+    for (int have = 2; have <= 8; have <<= 1) {
+        const int offset = 2 * have;                      // 4, 8, 16
+        const bool upper = (lane & offset) != 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (i < have) {
+                const float other = __shfl_xor_sync(0xffffffffu, a[i], offset);
+                a[i + have] = upper ? a[i] : other;
+                a[i] = upper ? other : a[i];
+            }
+        }
+    }
+}
+
+// Statistics (and logits) of 64 accumulator columns x 32 vocabulary rows held by a warp in the 16x256b layout:
+// va = rows 0-15 of the warp's lane quarter, vb = rows 16-31; this thread has rows g, g+8 (va) and g+16, g+24
+// (vb), g = lane / 4, and the 16 columns 8k + 2*(lane%4) + {0,1}.  Four rows of a column are reduced inside
+// the thread, the eight row groups by 14 exchanges - against 31 for 32 columns when every lane holds one row -
+// and column c's running statistic lives with the thread that owns it after the reduction (columns 2*lane and
+// 2*lane+1).  Rows are visited in ascending order across tiles, so an equal maximum later on never replaces
+// the index; the index work runs only when some column's maximum rises.
+__device__ __forceinline__ void stats_job64(const UmmaParams& p, uint32_t (&va)[32], uint32_t (&vb)[32], int lane, int quarter,
+                                            const TileCtx& tile, int tok0, int n_cols, float* run_m, float* run_s, int* run_i) {
+    const int g = lane >> 2, m4 = lane & 3;
     const bool greedy = p.greedy != 0;
-    // column maxima by a transposed butterfly (31 exchanges for 32 columns; a warp-wide reduction
-    // instruction per column measured ten times slower): lane l ends up with the maximum of column l
-    float mine_m;
-    {
-        float zc[32];
+    // rows of this thread: quarter * 32 + g + 8 h, h = 0..3
+    bool row_ok[4];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float z = (row_ok && j < n_cols) ? __uint_as_float(v[OFF + j]) : -INFINITY;
-            v[OFF + j] = __float_as_uint(z);
-            zc[j] = z;
+    for (int h = 0; h < 4; ++h) row_ok[h] = quarter * 32 + g + 8 * h < tile.rows;
+    const int vrow0 = tile.v0 + quarter * 32 + g;
+    // value (local column i = 2k + parity, row slot h): va/vb[4k + 2*(h&1) + parity]
+#define MASSV_VAL(i, h) ((h) < 2 ? va[4 * ((i) >> 1) + 2 * ((h) & 1) + ((i) & 1)] : vb[4 * ((i) >> 1) + 2 * ((h) & 1) + ((i) & 1)])
+    if (p.logits != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const int col = 8 * (i >> 1) + 2 * m4 + (i & 1);
+            if (col < n_cols && tok0 + col < p.M) {
+                float* dst = p.logits + (size_t)(tok0 + col) * p.V + vrow0;
+#pragma unroll
+                for (int h = 0; h < 4; ++h)
+                    if (row_ok[h]) dst[8 * h] = __uint_as_float(MASSV_VAL(i, h));
+            }
         }
-        transposed_max(zc, lane);
-        mine_m = zc[0];
     }
-    // Every column's maximum goes back to all lanes (it sits in lane j), which gives the lowest row attaining
-    // it and, at T > 0, the exponentials - without a branch per column (32 branches on a warp-uniform
-    // condition measured three times the cost of the whole butterfly).
-    const int warp_row0 = vrow - lane;          // vocabulary row of lane 0
-    int cand_idx = 0x7fffffff;
-    float mine_s = 0.f;
-    if (greedy) {
+    // 1. column maxima over the thread's rows (rows and columns that do not exist count as -inf)
+    float mx[16];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float mxj = __shfl_sync(0xffffffffu, mine_m, j);
-            const unsigned hit = __ballot_sync(0xffffffffu, __uint_as_float(v[OFF + j]) == mxj);
-            cand_idx = lane == j ? warp_row0 + (__ffs(hit) - 1) : cand_idx;
-        }
-    } else {
-        float sums[32];
+    for (int i = 0; i < 16; ++i) {
+        const bool col_ok = 8 * (i >> 1) + 2 * m4 + (i & 1) < n_cols;
+        float mi = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            const float mxj = __shfl_sync(0xffffffffu, mine_m, j);
-            const float z = __uint_as_float(v[OFF + j]);
-            const unsigned hit = __ballot_sync(0xffffffffu, z == mxj);
-            cand_idx = lane == j ? warp_row0 + (__ffs(hit) - 1) : cand_idx;
-            // (z - max) * scale as one multiply-add: -inf entries give 2^-inf = 0, an all -inf column is skipped below
-            sums[j] = exp2f(fmaf(z, p.scale_log2, -mxj * p.scale_log2));
+        for (int h = 0; h < 4; ++h) {
+            const float z = (row_ok[h] && col_ok) ? __uint_as_float(MASSV_VAL(i, h)) : -INFINITY;
+            MASSV_VAL(i, h) = __float_as_uint(z);
+            mi = fmaxf(mi, z);
         }
-        transposed_sum<32>(sums, lane);
-        mine_s = mine_m == -INFINITY ? 0.f : sums[0];
+        mx[i] = mi;
     }
-    const bool raise = mine_m > running.m;      // an equal maximum later on keeps the earlier (lower) index
-    const int new_idx = cand_idx;
-    if (raise) {
-        const float f = running.m == -INFINITY ? 0.f : exp2f((running.m - mine_m) * p.scale_log2);
-        running.s = greedy ? 0.f : mine_s + running.s * f;
-        running.m = mine_m;
-        running.idx = new_idx;
-    } else if (!greedy && mine_m != -INFINITY) {
-        running.s += mine_s * exp2f((mine_m - running.m) * p.scale_log2);
+    // 2. over the eight row groups: this thread ends up with the maxima of columns 2*lane, 2*lane+1
+    reduce_over_row_lanes(mx, lane, OpMax());
+    const int c_own = 2 * lane;                                // first owned column within the 64
+    float own_m[2] = {mx[0], mx[1]};
+    float old_m[2] = {run_m[c_own], run_m[c_own + 1]};
+    const bool raise0 = own_m[0] > old_m[0], raise1 = own_m[1] > old_m[1];
+    const bool any_raise = __any_sync(0xffffffffu, raise0 || raise1);
+    // 3. every thread needs the maxima of its 16 columns (for the index and for the exponentials)
+    if (any_raise || !greedy) gather_over_row_lanes(mx, lane);
+    int own_i[2] = {run_i[c_own], run_i[c_own + 1]};
+    if (any_raise) {
+        // lowest row attaining the maximum, per column: rows as floats (exact up to 2^24)
+        float cand[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            float c = 3.0e38f;
+#pragma unroll
+            for (int h = 3; h >= 0; --h)
+                if (__uint_as_float(MASSV_VAL(i, h)) == mx[i]) c = (float)(g + 8 * h);
+            cand[i] = c;
+        }
+        reduce_over_row_lanes(cand, lane, OpMin());
+        if (raise0) own_i[0] = tile.v0 + quarter * 32 + (int)cand[0];
+        if (raise1) own_i[1] = tile.v0 + quarter * 32 + (int)cand[1];
+    }
+    float own_s[2] = {0.f, 0.f};
+    if (!greedy) {
+        // 4. exponentials relative to the column's maximum in this tile, summed over the thread's rows, then over the row groups
+        float cs[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float bias = -mx[i] * p.scale_log2;
+            float acc = 0.f;
+#pragma unroll
+            for (int h = 0; h < 4; ++h) acc += exp2f(fmaf(__uint_as_float(MASSV_VAL(i, h)), p.scale_log2, bias));
+            cs[i] = mx[i] == -INFINITY ? 0.f : acc;            // an all -inf column would give NaN
+        }
+        reduce_over_row_lanes(cs, lane, OpAdd());
+        own_s[0] = cs[0]; own_s[1] = cs[1];
+    }
+#undef MASSV_VAL
+    // 5. fold into the running statistics of the two owned columns
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+        const int c = c_own + e;
+        if (c < n_cols) {
+            float rs = greedy ? 0.f : run_s[c];
+            if (e == 0 ? raise0 : raise1) {
+                const float f = old_m[e] == -INFINITY ? 0.f : exp2f((old_m[e] - own_m[e]) * p.scale_log2);
+                rs = greedy ? 0.f : own_s[e] + rs * f;
+                run_m[c] = own_m[e];
+                run_i[c] = own_i[e];
+            } else if (!greedy && own_m[e] != -INFINITY) {
+                rs += own_s[e] * exp2f((own_m[e] - old_m[e]) * p.scale_log2);
+            }
+            if (!greedy) run_s[c] = rs;
+        }
     }
 }
 
@@ -749,7 +799,6 @@ lm_head_duo_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_co
         // of a quarter take columns 64*part .. 64*part+63 of both sub-tiles.
         const int quarter = warp & 3;
         const int part = (warp - 2) >> 2;
-        const int row_in_tile = quarter * 32 + lane;
         const int c0 = part * 64;                              // first column (token row within the sub-tile)
         for (int c = threadIdx.x - 64; c < 4 * 2 * kDuoSubCols; c += kDuoEpilogueWarps * 32) {
             (&run_m[0][0])[c] = -INFINITY; (&run_s[0][0])[c] = 0.f; (&run_i[0][0])[c] = 0x7fffffff;
@@ -767,27 +816,22 @@ lm_head_duo_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_co
 #pragma unroll 1
             for (int q = 0; q < 2; ++q) {
                 // the sub-tile's 64 columns of this warp: into registers, and tensor memory is free for the next tile
-                uint32_t v[64];
+                uint32_t va[32], vb[32];
                 const bool live = (subs >> q) & 1;             // a half-tile computes one sub-tile only
                 if (live) {
-                    tmem_load64(taddr + q * kDuoSubCols, v);
-                    tmem_wait_ld<64>(v);
+                    tmem_load_16x64(taddr + q * kDuoSubCols, va);                              // rows 0-15 of the quarter
+                    tmem_load_16x64(taddr + q * kDuoSubCols + (16u << 16), vb);                // rows 16-31
+                    tmem_wait_ld<32>(va);
+                    tmem_wait_ld<32>(vb);
                 }
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_at(cluster_addr(&tmem_empty_bar[q], 0));
                 if (!live) continue;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int cc = c0 + h * 32;                // first column of the chunk within the sub-tile
-                    const int n_cols = min(32, sub - cc);
-                    if (n_cols > 0) {                           // the same in every lane
-                        const int col = q * kDuoSubCols + cc + lane;
-                        Stat running{run_m[quarter][col], run_s[quarter][col], run_i[quarter][col]};
-                        if (h == 0) stats_chunk32<0>(p, v, lane, row_in_tile, tile, q * sub + cc, n_cols, running);
-                        else stats_chunk32<32>(p, v, lane, row_in_tile, tile, q * sub + cc, n_cols, running);
-                        run_m[quarter][col] = running.m; run_s[quarter][col] = running.s; run_i[quarter][col] = running.idx;
-                    }
+                const int n_cols = min(64, sub - c0);
+                if (n_cols > 0) {                               // the same in every lane
+                    const int col = q * kDuoSubCols + c0;
+                    stats_job64(p, va, vb, lane, quarter, tile, q * sub + c0, n_cols, &run_m[quarter][col], &run_s[quarter][col], &run_i[quarter][col]);
                 }
             }
         }
