@@ -277,7 +277,8 @@ def roofline_block(kernel, bound, algorithmic, ms, peaks, peak_src, family):
 def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=None, want_e2e=False, want_tvd=False):
     """Generate one workload and time it: K steps bracketed by events on the launching stream, the L2
     flushed between steps; at least MIN_SPLIT_STEPS of them also carry the events that separate the
-    three calls and the ones the library records around its dominant kernels."""
+    three calls, and as many others the events the library records around its dominant kernels (kept
+    apart: an event between two kernels of a call keeps them from overlapping and costs a few us)."""
     import torch
     from workloads import generate, kv_bytes
     from paper_2505_10526_b200.binding import TIMED_ATTN, TIMED_LM_HEAD, TIMED_RESIDUAL
@@ -292,20 +293,23 @@ def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=Non
     sampling = cfg.temperature > 0
     n_ev = 10 if sampling else 8
 
-    def one_step(ev=None, split=False):
+    PLAIN, CALLS, KERNELS = 0, 1, 2
+
+    def one_step(ev=None, split=PLAIN):
         if ev:
             ev[0].record(stream)
-        if split:
+        if split == KERNELS:
             mv.massv_set_kernel_timing(TIMED_LM_HEAD, (ev[4], ev[5]))
             mv.massv_set_kernel_timing(TIMED_ATTN, (ev[6], ev[7]))
             if sampling:
                 mv.massv_set_kernel_timing(TIMED_RESIDUAL, (ev[8], ev[9]))
         step.attn(w)
-        if split:
+        if split == CALLS:
             ev[1].record(stream)
         step.accept(w)
-        if split:
+        if split == CALLS:
             ev[2].record(stream)
+        if split == KERNELS:
             for k in (TIMED_LM_HEAD, TIMED_ATTN, TIMED_RESIDUAL):
                 mv.massv_set_kernel_timing(k, None)
         step.commit(w["seq_lens"])
@@ -322,17 +326,21 @@ def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=Non
             e.record(stream)
         return evs
 
-    one_step(new_events(n_ev), split=True)             # the first instrumented step belongs to the warm-up
-    between_steps()
+    warm_ev = {}
+    for kind in (CALLS, KERNELS):                      # the first instrumented steps belong to the warm-up
+        warm_ev[kind] = new_events(n_ev)
+        one_step(warm_ev[kind], split=kind)
+        between_steps()
     for _ in range(max(W, 3)):
         one_step()
         between_steps()
     torch.cuda.synchronize()
     assert int(step.dev_status.item()) == 0, "device-side error during warm-up"
 
-    split_every = max(1, K // MIN_SPLIT_STEPS)
-    is_split = [i % split_every == 0 for i in range(K)]
-    events = [new_events(n_ev if is_split[i] else 4) for i in range(K)]
+    # every `period`-th step separates the calls, the step after it times the kernels, the rest are plain
+    period = max(2, K // MIN_SPLIT_STEPS)
+    is_split = [CALLS if i % period == 0 else KERNELS if i % period == 1 else PLAIN for i in range(K)]
+    events = [new_events(n_ev if is_split[i] == KERNELS else 4) for i in range(K)]
     launches0 = mv.massv_launch_count()
     barrier()
     torch.cuda.synchronize()
@@ -351,13 +359,15 @@ def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=Non
     assert int(step.dev_status.item()) == 0, "device-side error during the timed region"
 
     per_step = [e[0].elapsed_time(e[3]) for e in events]
-    sp = [e for e, s in zip(events, is_split) if s]
+    # (a run of a single step has no step of the other kind: the warm-up's stands in)
+    sp = [e for e, s in zip(events, is_split) if s == CALLS] or [warm_ev[CALLS]]
+    spk = [e for e, s in zip(events, is_split) if s == KERNELS] or [warm_ev[KERNELS]]
     t_attn = _stats([e[0].elapsed_time(e[1]) for e in sp])
     t_accept = _stats([e[1].elapsed_time(e[2]) for e in sp])
     t_commit = _stats([e[2].elapsed_time(e[3]) for e in sp])
-    t_lm = _stats([e[4].elapsed_time(e[5]) for e in sp])
-    t_attn_k = _stats([e[6].elapsed_time(e[7]) for e in sp])
-    t_res = _stats([e[8].elapsed_time(e[9]) for e in sp]) if sampling else None
+    t_lm = _stats([e[4].elapsed_time(e[5]) for e in spk])
+    t_attn_k = _stats([e[6].elapsed_time(e[7]) for e in spk])
+    t_res = _stats([e[8].elapsed_time(e[9]) for e in spk]) if sampling else None
     st = _stats(per_step)
     ms_per_step, value = aggregate_throughput(cfg.m, st["mean"], dev)
 
@@ -386,8 +396,9 @@ def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=Non
         "breakdown_ms": {"verify_attn": t_attn["mean"], "accept": t_accept["mean"], "kv_commit": t_commit["mean"],
                          "lm_head_kernel": t_lm["mean"], "attn_kernel": t_attn_k["mean"],
                          "residual_kernel": t_res["mean"] if sampling else None,
-                         "split_steps": len(sp),
-                         "note": "means over the timed steps that carry the extra events (they keep the kernels from overlapping)"},
+                         "split_steps": len(sp), "kernel_steps": len(spk),
+                         "note": "calls: means over the timed steps with an event between the calls; kernels: means over other "
+                                 "steps, in which the library records events around the kernel (no overlap with its neighbours)"},
         "rooflines": rl, "dominant": dominant, "share_of_step": {k: v / st["mean"] for k, v in shares.items()},
         "mean_accept_len": float(step.accept_len.float().mean()), "gpu_launches": int(launches),
         "wall_s_timed_region": wall, "mean_context": float(seq0.float().mean()),

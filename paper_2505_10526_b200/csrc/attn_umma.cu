@@ -11,9 +11,11 @@
 //   O[64, d]    += P[64, TILE] V_tile        V tile as TMA wrote it: [token][d] = MN-major B operand
 //
 // S (double buffered) and O live in tensor memory.  Warp roles: warp 0 streams K and V
-// tiles page by page with TMA into a ring and patches the block's own K/V rows into
-// the tiles that hold their positions (and stores them to their page slots: the
-// append); one thread of warp 1 issues the MMAs; warps 2-5 own 16 query rows each:
+// tiles page by page with TMA into a ring, and a pair's query rows (one box per block row:
+// the G heads of a KV head are adjacent) into one of two Q buffers ahead of the pair's first
+// tile; warp 6 (the helper) patches the block's own K/V rows into the tiles that hold their
+// positions (and stores them to their page slots: the append), so the stream of copies never
+// waits for a tile to land; one thread of warp 1 issues the MMAs; warps 2-5 own 16 query rows each:
 // they read S with tcgen05.ld (16x256b: the same fragment layout as a warp-level MMA
 // accumulator), apply scale, causal / window mask and the online softmax, and write P
 // as bf16 into shared memory for the second product.  O is rescaled in tensor memory
@@ -36,7 +38,11 @@ namespace massv {
 namespace {
 
 constexpr int kUmmaRows = 64;          // MMA M: query rows per KV head, padded
-constexpr int kUmmaThreads = 192;      // producer warp, MMA warp, four softmax warps
+// Warp 0: TMA producer; warp 1: MMA issuer and owner of the tensor-memory allocation; warps 2-5: softmax (warp w
+// reads TMEM lane quarter w % 4); warp 6: helper.  (Handing the softmax warps more registers with setmaxnreg -
+// roles regrouped so that they form one aligned group of four warps - measured 3 % slower on long contexts.)
+constexpr int kUmmaThreads = 224;
+constexpr int kProducerWarp = 0, kMmaWarp = 1, kHelperWarp = 6;
 constexpr int kUmmaMaxChunkPages = 256;
 constexpr int kFlatMaxBatch = 1024;    // sequences the flat schedule can index in shared memory
 constexpr float kRescaleThreshold = 8.f;   // log2 units
@@ -80,11 +86,11 @@ struct UmmaAttnCfg {
     static constexpr int kNCH = D / 64;                       // 64-element column groups of a K/V row
     static constexpr int kRegion = TILE * 128;                // bytes of one (TILE tokens x 64 elements) region
     static constexpr int kEntryBytes = kNCH * kRegion;        // one K tile or one V tile
-    static constexpr int kEntries = 5;                        // ring entries, filled in the order the MMAs consume them
+    static constexpr int kEntries = 4;                        // ring entries, filled in the order the MMAs consume them
     static constexpr int kQRegion = kUmmaRows * 128;          // (64 rows x 64 elements)
     static constexpr int kQBytes = kNCH * kQRegion;
     static constexpr int kPBytes = (TILE / 64) * kQRegion;    // P tile: 64 rows x TILE tokens, K-major
-    static constexpr int kSmem = kEntries * kEntryBytes + kQBytes + kPBytes + 1024;
+    static constexpr int kSmem = kEntries * kEntryBytes + 2 * kQBytes + kPBytes + 1024;      // Q is double buffered
     static constexpr int kColsNeeded = 2 * TILE + D;          // two S buffers and O
     static constexpr int kTmemCols = kColsNeeded <= 256 ? 256 : 512;
     static constexpr int kCtasPerSm = (kSmem <= 110 * 1024 && kTmemCols <= 256) ? 2 : 1;
@@ -121,7 +127,8 @@ struct Segment {
 
 template <int D, int TILE, bool FLAT>
 __global__ void __launch_bounds__(kUmmaThreads, UmmaAttnCfg<D, TILE>::kCtasPerSm)
-attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
+attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_q,
+                 const AttnParams p) {
     using Cfg = UmmaAttnCfg<D, TILE>;
     constexpr int E = Cfg::kEntries;
     constexpr int NCH = Cfg::kNCH;
@@ -138,7 +145,9 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     __shared__ __align__(8) uint64_t s_read_bar[2];    // S buffer copied to registers by the four softmax warps
     __shared__ __align__(8) uint64_t p_full_bar[2];    // P written by the four softmax warps
     __shared__ __align__(8) uint64_t pv_done_bar[2];   // P V of a tile done: P may be overwritten, O is up to date
-    __shared__ __align__(8) uint64_t q_ready_bar;      // the query rows of the next segment are in shared memory
+    __shared__ __align__(8) uint64_t q_ready_bar[2];   // the query rows of a segment are in shared memory (buffer = segment & 1)
+    __shared__ __align__(8) uint64_t q_free_bar[2];    // every score product of the segment that used the buffer is done
+    __shared__ __align__(8) uint64_t o_free_bar;       // the four softmax warps have read a finished segment's O
     __shared__ int s_cum[FLAT ? kFlatMaxBatch + 1 : 1];   // FLAT: tiles of sequences 0 .. b-1 (per KV head)
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
@@ -147,10 +156,28 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     const int G = p.Hq / p.Hkv;
     const int rows = G * p.R;
     const int rows_pad = (rows + 15) / 16 * 16;
+    // barriers and tensor memory do not depend on the kernel before this one
+    if (threadIdx.x == 0) {
+        for (int e = 0; e < E; ++e) { mbar_init(&ready_bar[e], 1); mbar_init(&landed_bar[e], 1); mbar_init(&empty_bar[e], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&s_full_bar[i], 1); mbar_init(&s_read_bar[i], 4); mbar_init(&p_full_bar[i], 4); mbar_init(&pv_done_bar[i], 1); }
+        mbar_init(&q_ready_bar[0], 1); mbar_init(&q_ready_bar[1], 1);
+        mbar_init(&q_free_bar[0], 1); mbar_init(&q_free_bar[1], 1);
+        mbar_init(&o_free_bar, 4);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {
+        __syncwarp();
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"((uint32_t)Cfg::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
     pdl_wait();
 
     // ---------------------------------------------------- this CTA's share of the work
     int f = 0, f_end = 0;                 // FLAT: range of the tile line; CHUNKED: one pseudo-tile
+    bool has_work = true;                 // a CTA without work still has to free its tensor memory
     if constexpr (FLAT) {
         // tiles per pair of every sequence, then an exclusive prefix sum over the batch
         for (int i = threadIdx.x; i < p.B; i += blockDim.x) {
@@ -189,18 +216,18 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         }
         f = min(total, (int)blockIdx.x * per_cta);
         f_end = min(total, f + per_cta);
-        if (f >= f_end) return;
+        has_work = f < f_end;
     } else {
         const int b = blockIdx.z, chunk = blockIdx.x;
         const int L = p.seq_lens[b];
         if (L < 0 || L + p.R > p.max_pages * kPageSize) {
             if (chunk == 0 && blockIdx.y == 0 && threadIdx.x == 0) set_status(p.dev_status, MASSV_ERR_CAPACITY);
-            return;
+            has_work = false;
+        } else {
+            const int lo_min = p.window > 0 ? max(0, L - p.window + 1) : 0;
+            has_work = chunk * p.kv_chunk < L + p.R && chunk >= lo_min / p.kv_chunk;
         }
-        if (chunk * p.kv_chunk >= L + p.R) return;
-        const int lo_min = p.window > 0 ? max(0, L - p.window + 1) : 0;
-        if (chunk < lo_min / p.kv_chunk) return;
-        f = 0; f_end = 1;
+        f = 0; f_end = has_work ? 1 : 0;
     }
     const int f_first = f;
     int b_hint = 0;
@@ -260,23 +287,15 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     };
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* q_smem = smem + E * Cfg::kEntryBytes;               // [NCH][64 rows][128 B], swizzled
-    uint8_t* p_smem = q_smem + Cfg::kQBytes;                     // [TILE/64][64 rows][128 B], swizzled
+    uint8_t* q_smem = smem + E * Cfg::kEntryBytes;               // two of [NCH][64 rows][128 B], swizzled
+    uint8_t* p_smem = q_smem + 2 * Cfg::kQBytes;                 // [TILE/64][64 rows][128 B], swizzled
+    // query rows past the last one are never copied: zero them once in both buffers
+    for (int i = threadIdx.x; i < 2 * (kUmmaRows - rows) * UPR; i += blockDim.x) {
+        const int buf = i / ((kUmmaRows - rows) * UPR), k = i % ((kUmmaRows - rows) * UPR), r = rows + k / UPR, u = k % UPR;
+        *reinterpret_cast<uint4*>(q_smem + buf * Cfg::kQBytes + (u / 8) * Cfg::kQRegion + swz128(r, u % 8)) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
-    if (threadIdx.x == 0) {
-        for (int e = 0; e < E; ++e) { mbar_init(&ready_bar[e], 1); mbar_init(&landed_bar[e], 1); mbar_init(&empty_bar[e], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&s_full_bar[i], 1); mbar_init(&s_read_bar[i], 4); mbar_init(&p_full_bar[i], 4); mbar_init(&pv_done_bar[i], 1); }
-        mbar_init(&q_ready_bar, 4);
-        abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 1) {
-        __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                     "r"((uint32_t)Cfg::kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -284,16 +303,34 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     const uint32_t tmem_o = tmem_base + 2 * TILE;
     volatile int* abort_ptr = &abort_flag;
     Segment sg;
-
-    if (warp == 0) {
-        // ------------------------------------------------ TMA producer (+ append / ragged-end patch)
+    if (!has_work) {
+        // nothing to compute: fall through to the release of tensor memory
+    } else if (warp == kProducerWarp) {
+        // ------------------------------------------------ TMA producer
         uint64_t policy;
         asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-        uint32_t landed_phase = 0;       // bit e: parity of the next completion of landed_bar[e]
         int it = 0;                      // items issued so far: ring entry it % E, use it / E
         bool ok = true;
-        while (ok && next_segment(sg)) {
+        for (int seg = 0; ok && next_segment(sg); ++seg) {
             const int n_tiles = sg.n_tiles, L = sg.L, b = sg.b, g = sg.g;
+            {
+                // Query rows of the pair, ahead of its tiles: row r = block_row * G + head_in_group, and the G heads of
+                // a block row are adjacent in memory, so a block row is one box per 64-element column group.  The
+                // buffer's last user is the segment before the previous one.
+                const int qb = seg & 1;
+                if (seg >= 2) {
+                    int fr = 0;
+                    if (lane == 0) fr = mbar_wait(&q_free_bar[qb], ((uint32_t)((seg - 2) >> 1)) & 1u, abort_ptr) ? 1 : 0;
+                    if (!__shfl_sync(0xffffffffu, fr, 0)) { ok = false; break; }
+                }
+                if (lane == 0) mbar_expect_tx(&q_ready_bar[qb], (uint32_t)(rows * D * 2));
+                __syncwarp();
+                for (int i = lane; i < p.R * NCH; i += 32) {
+                    const int j = i / NCH, dc = i % NCH;
+                    tma_load_2d(q_smem + qb * Cfg::kQBytes + dc * Cfg::kQRegion + j * G * 128, &map_q, dc * 64, (b * p.R + j) * p.Hq + g * G,
+                                &q_ready_bar[qb], policy);
+                }
+            }
             // Page ids travel in registers: lane l holds the id of page 32 * group + l of the segment, for
             // the group of the most advanced K tile (cur), the one before (prev: V tiles trail K tiles by up
             // to three tiles) and the one after (next: fetched a whole group ahead, so the table lookup is
@@ -302,16 +339,6 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             const int n_pages = (sg.c_end - sg.c_begin + kPageSize - 1) / kPageSize;
             int pid_prev = 0, pid_cur = lane < n_pages ? pt[lane] : 0, pid_next = 32 + lane < n_pages ? pt[32 + lane] : 0;
             int grp_cur = 0;
-            if (sg.c_end > L) {
-                // the segment ends with the block's own positions: bring the block's K/V rows into L2 now, so
-                // that the patches at its end do not each wait for a cold load
-                constexpr int LPR = D / 64;               // 128-byte lines per row
-                for (int i = lane; i < 2 * p.R * LPR; i += 32) {
-                    const int pv = i / (p.R * LPR), j = (i / LPR) % p.R, c = i % LPR;
-                    const __nv_bfloat16* src = (pv ? p.v_new : p.k_new) + (((size_t)b * p.R + j) * p.Hkv + g) * D + c * 64;
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
-                }
-            }
             for (int i = 0; i < 2 * n_tiles; ++i, ++it) {
                 // item i of the consumption order: which tile, and whether its K or its V
                 int t, is_v;
@@ -334,7 +361,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                 const int tile_start = sg.c_begin + t * TILE;
                 const int valid = min(TILE, sg.c_end - tile_start);
                 const int n_pg = (valid + kPageSize - 1) / kPageSize;
-                const bool patch = tile_start + TILE > L;           // the tile holds block rows or the ragged end
+                // a tile that holds block rows or the ragged end goes to the helper warp first
+                const bool patch = tile_start + TILE > L;
                 uint64_t* bar = patch ? &landed_bar[e] : &ready_bar[e];
                 uint8_t* dst = smem + (size_t)e * Cfg::kEntryBytes;
                 if (lane == 0) mbar_expect_tx(bar, (uint32_t)(n_pg * NCH * 2048));
@@ -347,26 +375,62 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                     if (pid < 0 || pid >= p.num_pages) { set_status(p.dev_status, MASSV_ERR_CAPACITY); pid = 0; }
                     tma_load_2d(dst + dc * Cfg::kRegion + pg * 2048, is_v ? &map_v : &map_k, dc * 64, (pid * p.Hkv + g) * kPageSize, bar, policy);
                 }
-                if (patch) {
-                    int landed = 0;
-                    if (lane == 0) landed = mbar_wait(&landed_bar[e], (landed_phase >> e) & 1u, abort_ptr) ? 1 : 0;
-                    landed = __shfl_sync(0xffffffffu, landed, 0);
-                    if (!landed) { ok = false; break; }
-                    landed_phase ^= 1u << e;
-                    // The block's rows (positions L .. L+gamma) are not in the cache yet: put them into the
-                    // tile and store them to their page slots.
+            }
+        }
+        if (lane == 0 && *abort_ptr) {
+            for (int i = 0; i < 64; ++i) __nanosleep(2000);   // let copies in flight land
+        }
+    } else if (warp == kHelperWarp) {
+        // ------------------------------------------------ helper: append / ragged-end patch
+        uint32_t landed_phase = 0;       // bit e: parity of the next completion of landed_bar[e]
+        int it_base = 0;                 // ring items of earlier segments
+        bool ok = true;
+        for (int seg = 0; ok && next_segment(sg); ++seg) {
+            const int n_tiles = sg.n_tiles, L = sg.L, b = sg.b, g = sg.g;
+            // ---- tiles that hold block rows (positions L .. L+gamma, not in the cache yet) or the ragged end: the
+            // rows go into the tile and to their page slots.  They are the last tiles of the segment; their items are
+            // taken in ring order, the rows fetched before the tile's own bytes are waited for.
+            if (sg.c_end > L) {
+                const int t_first = max(0, (L - sg.c_begin) / TILE);
+                const int32_t* pt = p.page_table + (size_t)b * p.max_pages;
+                for (int i = ring_item_of_k(t_first); i < 2 * n_tiles && ok; ++i) {
+                    int t, is_v;
+                    ring_item_decode(i, n_tiles, t, is_v);
+                    if (t < t_first) continue;
+                    const int e = (it_base + i) % E;
+                    const int tile_start = sg.c_begin + t * TILE;
+                    const int valid = min(TILE, sg.c_end - tile_start);
+                    uint8_t* dst = smem + (size_t)e * Cfg::kEntryBytes;
                     const int p_first = max(L, tile_start), p_last = min(sg.c_end, tile_start + TILE);
                     const __nv_bfloat16* src_base = is_v ? p.v_new : p.k_new;
                     __nv_bfloat16* pages = is_v ? p.v_pages : p.k_pages;
-                    for (int idx = lane; idx < (p_last - p_first) * UPR; idx += 32) {
-                        const int pos = p_first + idx / UPR, u = idx % UPR, row = pos - tile_start;
-                        const uint4 val = *reinterpret_cast<const uint4*>(src_base + (((size_t)b * p.R + (pos - L)) * p.Hkv + g) * D + u * 8);
-                        *reinterpret_cast<uint4*>(dst + (u / 8) * Cfg::kRegion + swz128(row, u % 8)) = val;
-                        int pid = tile_pid[0];
+                    const int n_units = (p_last - p_first) * UPR;
+                    constexpr int PRE = 4;                               // units per lane fetched ahead of the wait
+                    uint4 val[PRE];
+                    int pid[PRE];
 #pragma unroll
-                        for (int q = 1; q < PPT; ++q) pid = row / kPageSize == q ? tile_pid[q] : pid;
-                        if (pid >= 0 && pid < p.num_pages)
-                            *reinterpret_cast<uint4*>(pages + (((size_t)pid * p.Hkv + g) * kPageSize + (pos % kPageSize)) * D + u * 8) = val;
+                    for (int k = 0; k < PRE; ++k) {
+                        const int idx = k * 32 + lane;
+                        if (idx < n_units) {
+                            const int pos = p_first + idx / UPR, u = idx % UPR;
+                            val[k] = *reinterpret_cast<const uint4*>(src_base + (((size_t)b * p.R + (pos - L)) * p.Hkv + g) * D + u * 8);
+                            pid[k] = pt[pos / kPageSize];
+                        }
+                    }
+                    if (!mbar_wait_warp(&landed_bar[e], (landed_phase >> e) & 1u, abort_ptr)) { ok = false; break; }
+                    landed_phase ^= 1u << e;
+                    auto put = [&](int idx, const uint4& x, int page) {
+                        const int pos = p_first + idx / UPR, u = idx % UPR, row = pos - tile_start;
+                        *reinterpret_cast<uint4*>(dst + (u / 8) * Cfg::kRegion + swz128(row, u % 8)) = x;
+                        if (page >= 0 && page < p.num_pages)
+                            *reinterpret_cast<uint4*>(pages + (((size_t)page * p.Hkv + g) * kPageSize + (pos % kPageSize)) * D + u * 8) = x;
+                    };
+#pragma unroll
+                    for (int k = 0; k < PRE; ++k)
+                        if (k * 32 + lane < n_units) put(k * 32 + lane, val[k], pid[k]);
+                    for (int idx = PRE * 32 + lane; idx < n_units; idx += 32) {
+                        const int pos = p_first + idx / UPR, u = idx % UPR;
+                        put(idx, *reinterpret_cast<const uint4*>(src_base + (((size_t)b * p.R + (pos - L)) * p.Hkv + g) * D + u * 8), pt[pos / kPageSize]);
                     }
                     if (is_v) {
                         // rows past the end of the context hold stale bytes; their weights are zero, but
@@ -381,20 +445,19 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                     if (lane == 0) mbar_arrive(&ready_bar[e]);
                 }
             }
+            it_base += 2 * n_tiles;
         }
-        if (lane == 0 && *abort_ptr) {
-            for (int i = 0; i < 64; ++i) __nanosleep(2000);   // let copies in flight land
-        }
-    } else if (warp == 1) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(kUmmaRows, TILE, false);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(kUmmaRows, D, true);
-            const uint32_t q_lo = umma_desc_lo(smem_u32(q_smem));
+            uint32_t q_lo = umma_desc_lo(smem_u32(q_smem));
             const uint32_t p_lo = umma_desc_lo(smem_u32(p_smem));
             const uint32_t ring_addr = smem_u32(smem);
             bool ok = true;
             int it_base = 0, tau_base = 0, n_tiles = 0;      // ring items / tiles of earlier segments
+            int cur_seg = 0;
             // S[tau & 1] = Q K_t^T: d/16 steps of 16 elements (32 bytes) along the 128-byte rows
             auto issue_qk = [&](int t) {
                 const int i = it_base + ring_item_of_k(t), e = i % E, tau = tau_base + t;
@@ -411,6 +474,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                 }
                 umma_commit(&empty_bar[e]);
                 umma_commit(&s_full_bar[tau & 1]);
+                if (t == n_tiles - 1) umma_commit(&q_free_bar[cur_seg & 1]);      // the segment's last score product: its Q buffer is free
             };
             // O (+)= P V_t: TILE/16 steps of 16 tokens; V rows are tokens, so a step is 2048 bytes
             // further and the descriptor's leading offset is the distance between 64-element column groups
@@ -432,11 +496,19 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             };
             for (int seg = 0; ok && next_segment(sg); ++seg) {
                 n_tiles = sg.n_tiles;
-                // the softmax warps have read the previous segment's O and written this segment's Q
-                if (!mbar_wait(&q_ready_bar, (uint32_t)seg & 1u, abort_ptr)) { ok = false; break; }
+                cur_seg = seg;
+                // this segment's Q has landed in its buffer
+                if (!mbar_wait(&q_ready_bar[seg & 1], ((uint32_t)(seg >> 1)) & 1u, abort_ptr)) { ok = false; break; }
+                q_lo = umma_desc_lo(smem_u32(q_smem + (seg & 1) * Cfg::kQBytes));
                 tc_fence_after();
-                issue_qk(0);
-                if (ok && n_tiles > 1) issue_qk(1);
+                for (int t = 0; t < min(2, n_tiles) && ok; ++t) {
+                    // the S buffers still hold the last two tiles of the segment before until the softmax warps have read them
+                    const int tau = tau_base + t;
+                    if (tau >= 2 && !mbar_wait(&s_read_bar[tau & 1], ((uint32_t)((tau - 2) >> 1)) & 1u, abort_ptr)) { ok = false; break; }
+                    issue_qk(t);
+                }
+                // the first second product overwrites O: the softmax warps must have read the finished segment's
+                if (ok && seg > 0 && !mbar_wait(&o_free_bar, (uint32_t)(seg - 1) & 1u, abort_ptr)) { ok = false; break; }
                 for (int t = 0; t < n_tiles && ok; ++t) {
                     if (t + 2 < n_tiles) {
                         // S of tile t is in the softmax warps' registers: its buffer takes tile t+2.  Issued here,
@@ -460,26 +532,11 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
         // block row of each of this thread's two query rows (padding rows behave like the last block row)
         const int j0 = r0 < rows ? r0 / G : p.R - 1, j1 = r1 < rows ? r1 / G : p.R - 1;
         const float scale_log2 = p.scale * 1.4426950408889634f;
-        const int sm_tid = threadIdx.x - 64;                // 0 .. 127 among the softmax warps
         uint8_t* p_row0 = p_smem + r0 * 128 + 4 * (lane & 3);   // this thread's 4 bytes of unit 0 of row r0 (before the swizzle)
         bool ok = true;
         int tau_base = 0;
-        while (ok && next_segment(sg)) {
+        for (int seg = 0; ok && next_segment(sg); ++seg) {
             const int L = sg.L, b = sg.b, g = sg.g, n_tiles = sg.n_tiles, n_ctx = L + p.R;
-            // query rows of the pair (row r = block_row * G + head_in_group; rows past the last are zero).
-            // Every MMA that read the previous Q and every read of the previous O is finished by now.
-            for (int i = sm_tid; i < kUmmaRows * UPR; i += 128) {
-                const int r = i / UPR, u = i % UPR;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (r < rows)
-                    v = *reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.R + r / G) * p.Hq + g * G + r % G) * D + u * 8);
-                *reinterpret_cast<uint4*>(q_smem + (u / 8) * Cfg::kQRegion + swz128(r, u % 8)) = v;
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // Q is read by the tensor core
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&q_ready_bar);
-
             float m_ref[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
             for (int t = 0; t < n_tiles && ok; ++t) {
                 const int tau = tau_base + t, buf = tau & 1;
@@ -604,20 +661,21 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 1);
             l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], 2);
             const bool single = sg.part_o == nullptr;
-            const float inv0 = 1.f / l_run[0], inv1 = 1.f / l_run[1];
             const size_t out0 = r0 < rows ? (((size_t)b * p.R + r0 / G) * p.Hq + g * G + r0 % G) : 0;
             const size_t out1 = r1 < rows ? (((size_t)b * p.R + r1 / G) * p.Hq + g * G + r1 % G) : 0;
+            // (Each case has its own loop: this code runs once or twice per CTA, from a cold instruction cache,
+            // so what is not executed should not be fetched either.)
+            if (single) {
+                const float inv0 = 1.f / l_run[0], inv1 = 1.f / l_run[1];
 #pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 64) {
-                uint32_t o[32];
-                tmem_ld_16x64(tmem_o + lane_base + (uint32_t)c0, o);
+                for (int c0 = 0; c0 < D; c0 += 64) {
+                    uint32_t o[32];
+                    tmem_ld_16x64(tmem_o + lane_base + (uint32_t)c0, o);
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int c = c0 + k * 8 + 2 * (lane & 3);
-                    float a0 = __uint_as_float(o[4 * k + 0]), a1 = __uint_as_float(o[4 * k + 1]);
-                    float a2 = __uint_as_float(o[4 * k + 2]), a3 = __uint_as_float(o[4 * k + 3]);
-                    if (single) {
-                        a0 *= inv0; a1 *= inv0; a2 *= inv1; a3 *= inv1;
+                    for (int k = 0; k < 8; ++k) {
+                        const int c = c0 + k * 8 + 2 * (lane & 3);
+                        const float a0 = __uint_as_float(o[4 * k + 0]) * inv0, a1 = __uint_as_float(o[4 * k + 1]) * inv0;
+                        const float a2 = __uint_as_float(o[4 * k + 2]) * inv1, a3 = __uint_as_float(o[4 * k + 3]) * inv1;
                         if (r0 < rows) {
                             *reinterpret_cast<uint32_t*>(p.out + out0 * D + c) = pack_bf16x2(a0, a1);
                             if (p.out_f32) *reinterpret_cast<float2*>(p.out_f32 + out0 * D + c) = make_float2(a0, a1);
@@ -626,12 +684,41 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
                             *reinterpret_cast<uint32_t*>(p.out + out1 * D + c) = pack_bf16x2(a2, a3);
                             if (p.out_f32) *reinterpret_cast<float2*>(p.out_f32 + out1 * D + c) = make_float2(a2, a3);
                         }
-                    } else {
-                        if (r0 < rows) *reinterpret_cast<float2*>(sg.part_o + (size_t)r0 * D + c) = make_float2(a0, a1);
-                        if (r1 < rows) *reinterpret_cast<float2*>(sg.part_o + (size_t)r1 * D + c) = make_float2(a2, a3);
+                    }
+                }
+            } else if constexpr (FLAT) {
+                // A piece of a cut pair keeps the layout the accumulator has in registers: unit
+                // ((qd * D/64 + c0/64) * 8 + k) * 32 + lane is one 16-byte store of (row r0: columns c, c+1; row r1:
+                // the same columns), c = c0 + 8k + 2 (lane % 4).  The merge kernel reads it back the same way.
+                if (qd * 16 < rows) {
+                    float4* dst = reinterpret_cast<float4*>(sg.part_o) + (size_t)(qd * NCH) * 8 * 32 + lane;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < D; c0 += 64) {
+                        uint32_t o[32];
+                        tmem_ld_16x64(tmem_o + lane_base + (uint32_t)c0, o);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            dst[((c0 / 64) * 8 + k) * 32] = make_float4(__uint_as_float(o[4 * k + 0]), __uint_as_float(o[4 * k + 1]),
+                                                                        __uint_as_float(o[4 * k + 2]), __uint_as_float(o[4 * k + 3]));
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int c0 = 0; c0 < D; c0 += 64) {
+                    uint32_t o[32];
+                    tmem_ld_16x64(tmem_o + lane_base + (uint32_t)c0, o);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const int c = c0 + k * 8 + 2 * (lane & 3);
+                        if (r0 < rows) *reinterpret_cast<float2*>(sg.part_o + (size_t)r0 * D + c) = make_float2(__uint_as_float(o[4 * k + 0]), __uint_as_float(o[4 * k + 1]));
+                        if (r1 < rows) *reinterpret_cast<float2*>(sg.part_o + (size_t)r1 * D + c) = make_float2(__uint_as_float(o[4 * k + 2]), __uint_as_float(o[4 * k + 3]));
                     }
                 }
             }
+            // O is in registers or on its way to memory: the next segment's second product may overwrite it
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_free_bar);
             if ((lane & 3) == 0) {
                 if (single) {
                     if (p.lse) {
@@ -649,7 +736,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     pdl_trigger();
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)Cfg::kTmemCols) : "memory");
@@ -657,15 +744,17 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
     if (threadIdx.x == 0 && abort_flag) set_status(p.dev_status, MASSV_ERR_TIMEOUT);
 }
 
-// Merge the pieces of every (sequence, KV head) pair that the flat schedule cut: one CTA per pair,
-// all of its query rows.  The pieces of a pair sit in consecutive CTAs of the split kernel; piece c is
-// in slot 0 of CTA c unless the pair begins inside that CTA's range.  Pieces are summed in order.
+// Merge the pieces of every (sequence, KV head) pair that the flat schedule cut.  The pieces of a pair sit in
+// consecutive CTAs of the split kernel; piece c is in slot 0 of CTA c unless the pair begins inside that CTA's
+// range.  A piece has the layout of the accumulator in registers (see the split kernel): unit
+// ((qd * d/64 + ch) * 8 + k) * 32 + lane holds rows qd*16 + lane/4 (.x, .y) and +8 (.z, .w), columns
+// ch*64 + 8k + 2*(lane%4) + {0, 1}.  grid (pair, qd * parts + part): a CTA merges `units_per_cta` units of one
+// group of 16 rows, so it needs the weights of those rows only.  Pieces are summed in a fixed order.
 constexpr int kFlatCombineThreads = 256;
-__global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(const AttnParams p, int rows_pad, int rows_per_cta) {
-    const int G = p.Hq / p.Hkv;
+__global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(const AttnParams p, int rows_pad, int parts, int units_per_cta) {
+    const int G = p.Hq / p.Hkv, rows = G * p.R;
     const int g = blockIdx.x % p.Hkv, b = blockIdx.x / p.Hkv;
-    // with few pairs each pair's rows are dealt to several CTAs (blockIdx.y)
-    const int row0 = blockIdx.y * rows_per_cta, rows = min(rows_per_cta, G * p.R - row0);
+    const int qd = blockIdx.y / parts, part = blockIdx.y % parts;
     pdl_wait();
     pdl_trigger();
     const int per_cta = p.flat_meta[0];
@@ -676,97 +765,89 @@ __global__ void __launch_bounds__(kFlatCombineThreads) attn_flat_combine_kernel(
     if (c_first == c_last) return;                 // the pair was finished by one CTA
     const int n = c_last - c_first + 1;
     auto slot_of = [&](int i) -> size_t { const int c = c_first + i; return (size_t)c * 2 + (start <= c * per_cta ? 0 : 1); };
-    // per row: the common maximum and 1 / sum; per (piece, row): the merge weight
     extern __shared__ float4 s_red[];              // [kFlatCombineThreads]: partial sums of the piece groups (below)
-    float* s_comb = reinterpret_cast<float*>(s_red + kFlatCombineThreads);
-    float* s_w = s_comb;                           // [n][rows]: first the piece maxima, then the merge weights
-    float* s_l = s_comb + (size_t)n * rows;        // [n][rows]: the pieces' sums
-    float* s_inv = s_comb + 2 * (size_t)n * rows;  // [rows]
+    float* s_w = reinterpret_cast<float*>(s_red + kFlatCombineThreads);   // [n][16]: first the piece maxima, then the merge weights
+    float* s_l = s_w + (size_t)n * 16;             // [n][16]: the pieces' sums
+    float* s_inv = s_l + (size_t)n * 16;           // [16]
     // every (piece, row) pair's (max, sum) with one load per thread: a pair cut into dozens of pieces
     // must not walk them one latency after the other
-    for (int idx = threadIdx.x; idx < n * rows; idx += blockDim.x) {
-        const int i = idx / rows, rr = idx % rows;
-        const float2 ml = *reinterpret_cast<const float2*>(p.flat_part_ml + (slot_of(i) * rows_pad + row0 + rr) * 2);
+    for (int idx = threadIdx.x; idx < n * 16; idx += blockDim.x) {
+        const int i = idx / 16, r = qd * 16 + idx % 16;
+        float2 ml = make_float2(-INFINITY, 0.f);
+        if (r < rows) ml = *reinterpret_cast<const float2*>(p.flat_part_ml + (slot_of(i) * rows_pad + r) * 2);
         s_w[idx] = ml.x;
         s_l[idx] = ml.y;
     }
     __syncthreads();
-    for (int rr = threadIdx.x; rr < rows; rr += blockDim.x) {
-        const int r = row0 + rr;
+    if (threadIdx.x < 16) {
+        const int rr = threadIdx.x, r = qd * 16 + rr;
         float M = -INFINITY;
-        for (int i = 0; i < n; ++i) M = fmaxf(M, s_w[(size_t)i * rows + rr]);
+        for (int i = 0; i < n; ++i) M = fmaxf(M, s_w[i * 16 + rr]);
         float Lsum = 0.f;
         for (int i = 0; i < n; ++i) {
-            const float mi = s_w[(size_t)i * rows + rr];
+            const float mi = s_w[i * 16 + rr];
             const float w = mi == -INFINITY ? 0.f : exp2f(mi - M);
-            s_w[(size_t)i * rows + rr] = w;
-            Lsum += s_l[(size_t)i * rows + rr] * w;
+            s_w[i * 16 + rr] = w;
+            Lsum += s_l[i * 16 + rr] * w;
         }
         s_inv[rr] = 1.f / Lsum;
-        if (p.lse) p.lse[((size_t)b * p.R + r / G) * p.Hq + g * G + r % G] = (M + log2f(Lsum)) * 0.6931471805599453f;
+        if (p.lse && part == 0 && r < rows) p.lse[((size_t)b * p.R + r / G) * p.Hq + g * G + r % G] = (M + log2f(Lsum)) * 0.6931471805599453f;
     }
     __syncthreads();
-    const int quads = p.d / 4;                     // a thread produces four channels of one row at a time
-    auto store_row = [&](int rr, int c, float4 acc) {
-        const int r = row0 + rr;
-        const float inv = s_inv[rr];
-        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        const size_t row_out = ((size_t)b * p.R + r / G) * p.Hq + g * G + r % G;
-        uint2 packed;
-        packed.x = pack_bf16x2(acc.x, acc.y);
-        packed.y = pack_bf16x2(acc.z, acc.w);
-        *reinterpret_cast<uint2*>(p.out + row_out * p.d + c) = packed;
-        if (p.out_f32) *reinterpret_cast<float4*>(p.out_f32 + row_out * p.d + c) = acc;
+    const int nch = p.d / 64;
+    const int unit0 = qd * nch * 256 + part * units_per_cta;       // first unit of this CTA within a piece
+    const float4* pieces = reinterpret_cast<const float4*>(p.flat_part_o);
+    const size_t piece_units = (size_t)rows_pad * p.d / 4;
+    auto store_unit = [&](int idx, float4 acc) {
+        const int u = part * units_per_cta + idx;                   // unit within the row group
+        const int lane = u % 32, k = (u / 32) % 8, ch = u / 256;
+        const int rr = lane / 4, c = ch * 64 + k * 8 + 2 * (lane % 4);
+        const float i0 = s_inv[rr], i1 = s_inv[rr + 8];
+        acc.x *= i0; acc.y *= i0; acc.z *= i1; acc.w *= i1;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int r = qd * 16 + rr + 8 * h;
+            if (r < rows) {
+                const size_t row_out = ((size_t)b * p.R + r / G) * p.Hq + g * G + r % G;
+                const float x = h ? acc.z : acc.x, y = h ? acc.w : acc.y;
+                *reinterpret_cast<uint32_t*>(p.out + row_out * p.d + c) = pack_bf16x2(x, y);
+                if (p.out_f32) *reinterpret_cast<float2*>(p.out_f32 + row_out * p.d + c) = make_float2(x, y);
+            }
+        }
     };
-    // Few outputs and many pieces (a short batch cut across the whole grid): several threads share an
-    // output, thread group k summing pieces k, k + groups, ... with all its loads in flight at once; the
-    // groups' sums are then added in group order.  The order of the sums is fixed, so results repeat.
-    const int want = rows * quads, groups = (int)blockDim.x / want;
+    auto add_piece = [&](float4& acc, int i, int idx) {
+        const float4 v = pieces[slot_of(i) * piece_units + unit0 + idx];
+        const int rr = ((part * units_per_cta + idx) % 32) / 4;
+        const float w0 = s_w[i * 16 + rr], w1 = s_w[i * 16 + rr + 8];
+        acc.x += v.x * w0; acc.y += v.y * w0; acc.z += v.z * w1; acc.w += v.w * w1;
+    };
+    // Few units and many pieces (a short batch cut across the whole grid): several threads share a unit,
+    // thread group k summing pieces k, k + groups, ... with all its loads in flight at once; the groups'
+    // sums are then added in group order.  The order of the sums is fixed, so results repeat.
+    const int groups = (int)blockDim.x / units_per_cta;
     if (groups >= 2 && n >= 4) {
-        const int grp = threadIdx.x / want, idx = threadIdx.x % want;
-        const int rr = idx / quads, r = row0 + rr, c = (idx % quads) * 4;
+        const int grp = threadIdx.x / units_per_cta, idx = threadIdx.x % units_per_cta;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         if (grp < groups) {
 #pragma unroll 4
-            for (int i = grp; i < n; i += groups) {
-                const float4 v = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i) * rows_pad + r) * p.d + c);
-                const float w = s_w[(size_t)i * rows + rr];
-                acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
-            }
+            for (int i = grp; i < n; i += groups) add_piece(acc, i, idx);
             s_red[threadIdx.x] = acc;
         }
         __syncthreads();
         if (grp == 0) {
             for (int k = 1; k < groups; ++k) {
-                const float4 v = s_red[k * want + idx];
+                const float4 v = s_red[k * units_per_cta + idx];
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
             }
-            store_row(rr, c, acc);
+            store_unit(idx, acc);
         }
         return;
     }
-    for (int idx = threadIdx.x; idx < rows * quads; idx += blockDim.x) {
-        const int rr = idx / quads, r = row0 + rr, c = (idx % quads) * 4;
+    for (int idx = threadIdx.x; idx < units_per_cta; idx += blockDim.x) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        int i = 0;
-        for (; i + 4 <= n; i += 4) {                // four independent loads in flight, summed in piece order
-            const float4 v0 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i) * rows_pad + r) * p.d + c);
-            const float4 v1 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i + 1) * rows_pad + r) * p.d + c);
-            const float4 v2 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i + 2) * rows_pad + r) * p.d + c);
-            const float4 v3 = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i + 3) * rows_pad + r) * p.d + c);
-            const float w0 = s_w[(size_t)i * rows + rr], w1 = s_w[(size_t)(i + 1) * rows + rr];
-            const float w2 = s_w[(size_t)(i + 2) * rows + rr], w3 = s_w[(size_t)(i + 3) * rows + rr];
-            acc.x += v0.x * w0; acc.y += v0.y * w0; acc.z += v0.z * w0; acc.w += v0.w * w0;
-            acc.x += v1.x * w1; acc.y += v1.y * w1; acc.z += v1.z * w1; acc.w += v1.w * w1;
-            acc.x += v2.x * w2; acc.y += v2.y * w2; acc.z += v2.z * w2; acc.w += v2.w * w2;
-            acc.x += v3.x * w3; acc.y += v3.y * w3; acc.z += v3.z * w3; acc.w += v3.w * w3;
-        }
-        for (; i < n; ++i) {
-            const float4 v = *reinterpret_cast<const float4*>(p.flat_part_o + (slot_of(i) * rows_pad + r) * p.d + c);
-            const float w = s_w[(size_t)i * rows + rr];
-            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
-        }
-        store_row(rr, c, acc);
+#pragma unroll 4
+        for (int i = 0; i < n; ++i) add_piece(acc, i, idx);      // summed in piece order, four loads in flight
+        store_unit(idx, acc);
     }
 }
 
@@ -783,6 +864,9 @@ template <int D, int TILE>
 cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtensorMap& mv, cudaStream_t stream, bool flat, int* launched,
                         cudaEvent_t split_done) {
     using Cfg = UmmaAttnCfg<D, TILE>;
+    // the query rows as a [B * R * Hq, D] matrix; a box is the G adjacent heads of one block row
+    CUtensorMap mq;
+    if (!make_tensor_map_bf16_2d(&mq, p.q, (uint64_t)p.B * p.R * p.Hq, D, (uint32_t)(p.Hq / p.Hkv))) return cudaErrorInvalidValue;
     static_assert(Cfg::kColsNeeded <= 512, "S buffers and O fit tensor memory");
     static_assert(Cfg::kSmem <= 227 * 1024, "ring, Q and P fit shared memory");
     cudaError_t e;
@@ -791,30 +875,28 @@ cudaError_t launch_umma(const AttnParams& p, const CUtensorMap& mk, const CUtens
         if (e != cudaSuccess) return e;
         int ctas = flat_sm_count() * Cfg::kCtasPerSm;
         if (ctas > kFlatMaxCtas) ctas = kFlatMaxCtas;
-        e = launch_pdl(attn_umma_kernel<D, TILE, true>, dim3(ctas), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, p);
+        e = launch_pdl(attn_umma_kernel<D, TILE, true>, dim3(ctas), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, mq, p);
         if (e != cudaSuccess) return e;
         if (split_done && cudaEventRecord(split_done, stream) != cudaSuccess) return cudaGetLastError();
         const int rows = (p.Hq / p.Hkv) * p.R;
-        // (max, sum) and weight for at most `ctas` pieces of a pair (a pair can span every CTA), plus one value per row
-        // enough CTAs to fill the machine: a pair's rows are dealt to several CTAs when there are few pairs
-        const int pairs = p.B * p.Hkv;
-        int row_groups = (2 * flat_sm_count() + pairs - 1) / pairs;
-        if (row_groups > rows) row_groups = rows;
-        const int rows_per_cta = (rows + row_groups - 1) / row_groups;
-        row_groups = (rows + rows_per_cta - 1) / rows_per_cta;
-        const size_t comb_smem = (2 * (size_t)ctas + 1) * rows_per_cta * sizeof(float) + kFlatCombineThreads * sizeof(float4);
+        // enough CTAs to fill the machine: a pair's groups of 16 rows go to separate CTAs, and with few pairs a
+        // group's units (D/64 * 256 of them) are cut further into 2, 4, 8 or 16 parts
+        const int pairs = p.B * p.Hkv, rows_pad = attn_rows_pad(rows), n_qd = rows_pad / 16, units_per_qd = (D / 64) * 256;
+        int parts = 1;
+        while (parts < 16 && units_per_qd / (parts * 2) >= 32 && pairs * n_qd * parts < 2 * flat_sm_count()) parts *= 2;
+        // (max, sum) and weight of 16 rows for at most `ctas` pieces of a pair (a pair can span every CTA)
+        const size_t comb_smem = (2 * (size_t)ctas + 1) * 16 * sizeof(float) + kFlatCombineThreads * sizeof(float4);
         e = cudaFuncSetAttribute(attn_flat_combine_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)comb_smem);
         if (e != cudaSuccess) return e;
-        // with few outputs per CTA the spare threads share the pieces of an output (see the kernel)
-        const int threads = kFlatCombineThreads;
-        e = launch_pdl(attn_flat_combine_kernel, dim3(pairs, row_groups), dim3(threads), comb_smem, stream, p, attn_rows_pad(rows), rows_per_cta);
+        e = launch_pdl(attn_flat_combine_kernel, dim3(pairs, n_qd * parts), dim3(kFlatCombineThreads), comb_smem, stream, p, rows_pad, parts,
+                       units_per_qd / parts);
         *launched = 2;
         return e;
     }
     e = cudaFuncSetAttribute(attn_umma_kernel<D, TILE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmem);
     if (e != cudaSuccess) return e;
     *launched = 1;
-    return launch_pdl(attn_umma_kernel<D, TILE, false>, dim3(p.max_chunks, p.Hkv, p.B), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, p);
+    return launch_pdl(attn_umma_kernel<D, TILE, false>, dim3(p.max_chunks, p.Hkv, p.B), dim3(kUmmaThreads), (size_t)Cfg::kSmem, stream, mk, mv, mq, p);
 }
 
 }  // namespace
