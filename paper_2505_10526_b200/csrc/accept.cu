@@ -224,42 +224,46 @@ __device__ __forceinline__ double block_total(double x, double* smem_warp) {
     return tot;
 }
 
-// Block-wide exclusive prefix of one double per thread, in thread order; *total gets the sum.
-__device__ __forceinline__ double block_exclusive_scan(double x, double* smem_warp, double* total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    double incl = x;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double y = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += y;
-    }
-    if (lane == 31) smem_warp[warp] = incl;
-    bar_sync_consumers();
-    double base = 0.0, tot = 0.0;
-    for (int w = 0; w < kSampleThreads / 32; ++w) {
-        const double s = smem_warp[w];
-        if (w < warp) base += s;
-        tot += s;
-    }
-    bar_sync_consumers();
-    *total = tot;
-    return base + incl - x;
-}
-
 // Inside the chunk that holds the target: the first entry (in vocabulary order) whose running mass
 // exceeds `target`, starting from `base`, and the last entry with positive mass.  r as produced by
 // masses_of.  Results through s_first / s_last (shared), valid after the call for every thread.
+// The four quarters of the chunk are scanned together (one pass of shuffles, two barriers); scratch holds
+// 4 doubles per warp.
+constexpr int kPickScratch = 4 * (kSampleThreads / 32);
 __device__ __forceinline__ void pick_in_chunk(const float (&r)[kPerThread], int chunk_first_entry, double base, double target,
-                                              double* smem_warp, int* s_first, int* s_last) {
-    const int t = threadIdx.x;
+                                              double* scratch, int* s_first, int* s_last) {
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     if (t == 0) { *s_first = 0x7fffffff; *s_last = -1; }
+    double g[4], incl[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {            // quarter j of the chunk: groups 256 j .. 256 j + 255, one per thread
+        g[j] = ((double)r[4 * j] + (double)r[4 * j + 1]) + ((double)r[4 * j + 2] + (double)r[4 * j + 3]);
+        incl[j] = g[j];
+    }
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const double y = __shfl_up_sync(0xffffffffu, incl[j], o);
+            if (lane >= o) incl[j] += y;
+        }
+    }
+    if (lane == 31) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) scratch[warp * 4 + j] = incl[j];
+    }
+    bar_sync_consumers();
     int first = 0x7fffffff, last = -1;
     double run_base = base;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {            // quarter j of the chunk: groups 256 j .. 256 j + 255, one per thread
-        const double g = ((double)r[4 * j] + (double)r[4 * j + 1]) + ((double)r[4 * j + 2] + (double)r[4 * j + 3]);
-        double quarter;
-        double run = run_base + block_exclusive_scan(g, smem_warp, &quarter);
+    for (int j = 0; j < 4; ++j) {
+        double warp_base = 0.0, quarter = 0.0;              // the warps' totals in warp order
+        for (int w = 0; w < kSampleThreads / 32; ++w) {
+            const double s = scratch[w * 4 + j];
+            if (w < warp) warp_base += s;
+            quarter += s;
+        }
+        double run = run_base + (warp_base + incl[j] - g[j]);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             run += (double)r[4 * j + e];
@@ -271,17 +275,59 @@ __device__ __forceinline__ void pick_in_chunk(const float (&r)[kPerThread], int 
         }
         run_base += quarter;
     }
-    bar_sync_consumers();
     atomicMin(s_first, first);
     atomicMax(s_last, last);
     bar_sync_consumers();
 }
 
-__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(smem_u32(dst)),
-        "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
-        : "memory");
+// The sequential part of a draw, by one warp: n chunk masses (shared memory, vocabulary order) -> the chunk that
+// holds u * total, the mass before it, and whether rounding pushed the target past the last positive chunk.  Lane l
+// sums a contiguous run of chunks, a shuffle scan adds the lanes up (a fixed order), and the lowest lane whose
+// run crosses the target wins.  s_pick[0] = chunk (-1: no mass at all), s_pick[1] = take the last positive entry,
+// s_base[0] = mass before the chunk, s_base[1] = target.
+__device__ __forceinline__ void walk_chunk_masses(const double* s, int n, double u, int* s_pick, double* s_base) {
+    const int lane = threadIdx.x & 31;
+    const int per = (n + 31) / 32;
+    const int i0 = min(n, lane * per), i1 = min(n, i0 + per);
+    double local = 0.0;
+    for (int i = i0; i < i1; ++i) local += s[i];
+    double incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    const double tot = __shfl_sync(0xffffffffu, incl, 31);
+    const double target = u * tot;
+    double run = incl - local, my_base = 0.0;
+    int my_pick = 0x7fffffff, my_last = -1;
+    for (int i = i0; i < i1; ++i) {
+        const double sm = s[i];
+        if (sm > 0.0) {
+            my_last = i;
+            if (my_pick == 0x7fffffff && run + sm > target) { my_pick = i; my_base = run; }
+        }
+        run += sm;
+    }
+    const unsigned found = __ballot_sync(0xffffffffu, my_pick != 0x7fffffff);
+    const int last_pos = __reduce_max_sync(0xffffffffu, my_last);
+    const int src = found ? __ffs(found) - 1 : 0;
+    const int pick = __shfl_sync(0xffffffffu, my_pick, src);
+    const double base = __shfl_sync(0xffffffffu, my_base, src);
+    if (lane == 0) {
+        s_pick[0] = tot > 0.0 ? (found ? pick : last_pos) : -1;
+        s_pick[1] = found ? 0 : 1;
+        s_base[0] = found ? base : 0.0;
+        s_base[1] = target;
+    }
+}
+
+// (No eviction hint: the chunk that turns out to hold the drawn token is read a second time, and should then
+// still be in L2.)
+__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)), "l"(src),
+                 "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
 }
 
 // The sequential part of the draw for one sequence, by the 256 threads of warps 0-7: walk the chunk masses
@@ -302,14 +348,16 @@ __device__ void draw_from_chunk_masses(const AcceptParams& p, int b, const SeqSt
             for (int i = t; i < p.n_chunks; i += kSampleThreads) s_sums[i] = __ldcg(sums + i);
             bar_sync_consumers();
         }
-        if (t == 0) {
+        if (staged) {
+            if (t < 32) walk_chunk_masses(s_sums, p.n_chunks, (double)p.u_sample[(size_t)b * R + st.n], s_pick, s_base);
+        } else if (t == 0) {
             double tot = 0.0;
-            for (int i = 0; i < p.n_chunks; ++i) tot += staged ? s_sums[i] : ((volatile double*)sums)[i];
+            for (int i = 0; i < p.n_chunks; ++i) tot += ((volatile double*)sums)[i];
             const double target = (double)p.u_sample[(size_t)b * R + st.n] * tot;
             int pick = -1, last_pos = -1;
             double cum = 0.0, base = 0.0;
             for (int i = 0; i < p.n_chunks; ++i) {
-                const double sm = staged ? s_sums[i] : ((volatile double*)sums)[i];
+                const double sm = ((volatile double*)sums)[i];
                 if (sm > 0.0) last_pos = i;
                 if (pick < 0 && sm > 0.0 && cum + sm > target) { pick = i; base = cum; }
                 cum += sm;
@@ -361,7 +409,7 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
     __shared__ __align__(8) uint64_t full_bar[kResidualStages];     // the item's bytes have landed
     __shared__ __align__(8) uint64_t done_bar[kResidualStages];     // the eight consumer warps are done with the stage
     __shared__ double s_part[kResidualStages][kSampleThreads / 32];
-    __shared__ double warp_sums[kSampleThreads / 32];
+    __shared__ double warp_sums[kPickScratch];
     __shared__ double s_sums[kWalkChunks];
     __shared__ SeqState s_state[kResidualSeqCache];
     __shared__ int s_pending[kResidualSeqCache], s_n_pending;
@@ -388,7 +436,12 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
     if (n_items <= 0) return;
     {
         const int n_seq = (i1 - 1) / p.n_chunks - b_lo + 1;
-        if (t < min(n_seq, kResidualSeqCache)) s_state[t] = p.seq_state[b_lo + t];
+        if (t < min(n_seq, kResidualSeqCache)) {
+            const SeqState st = p.seq_state[b_lo + t];
+            s_state[t] = st;
+            // the uniform of the draw is read at the very end, by whichever CTA completes the sequence: into L2 now
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(p.u_sample + (size_t)(b_lo + t) * R + st.n));
+        }
     }
     __syncthreads();
     auto state_of = [&](int b) -> SeqState { return b - b_lo < kResidualSeqCache ? s_state[b - b_lo] : p.seq_state[b]; };
@@ -398,8 +451,6 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
     if (warp == kSampleThreads / 32) {
         // ------------------------------------------------ producer
         if (lane == 0) {
-            uint64_t policy;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
             int run_cnt = 0;               // chunks of the current sequence finished since this CTA's last arrival
             bool ok = true;
             for (int k = 0; k < n_items + kResidualStages && ok; ++k) {
@@ -417,7 +468,10 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
                         const unsigned prev = atomicAdd(&p.counters[b], (unsigned)run_cnt);
                         if (prev + (unsigned)run_cnt == (unsigned)p.n_chunks) {
                             // every chunk of b is in: the draw is this CTA's (its slot in the list is free: a CTA
-                            // completes at most one sequence per sequence it holds items of)
+                            // completes at most one sequence per sequence it holds items of).  The fence orders the
+                            // other CTAs' masses, stored before their arrivals, ahead of this CTA's reads of them
+                            // (which follow the barrier below).
+                            __threadfence();
                             if (s_n_pending < kResidualSeqCache) s_pending[s_n_pending++] = b;
                             else set_status(p.dev_status, MASSV_ERR_UNSUPPORTED);
                         }
@@ -430,10 +484,10 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
                     const uint32_t bytes = (uint32_t)min(kResidualChunk, p.V - c * kResidualChunk) * 4u;
                     uint8_t* dst = res_smem + (size_t)s * kStageBytes;
                     mbar_expect_tx(&full_bar[s], st.use_q ? 2 * bytes : bytes);
-                    bulk_load_1d(dst, p.logits + (size_t)(b * R + st.n) * p.V + (size_t)c * kResidualChunk, bytes, &full_bar[s], policy);
+                    bulk_load_1d(dst, p.logits + (size_t)(b * R + st.n) * p.V + (size_t)c * kResidualChunk, bytes, &full_bar[s]);
                     if (st.use_q)
                         bulk_load_1d(dst + kResidualChunk * 4, p.draft_probs + ((size_t)b * p.gamma + st.n) * p.V + (size_t)c * kResidualChunk,
-                                     bytes, &full_bar[s], policy);
+                                     bytes, &full_bar[s]);
                 }
             }
         }
@@ -484,7 +538,6 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
     if (warp == kSampleThreads / 32) return;
     const int n_pending = s_n_pending;
     for (int i = 0; i < n_pending; ++i) {
-        __threadfence();           // the other CTAs' chunk masses, counted before this CTA's arrival
         const int b = s_pending[i];
         draw_from_chunk_masses(p, b, state_of(b), inv_T, warp_sums, s_sums, s_pick, s_base, &s_first, &s_last);
     }
@@ -548,7 +601,7 @@ __global__ void __launch_bounds__(kSampleThreads) shard_pick_kernel(ShardParams 
     pdl_wait();
     pdl_trigger();
     const SeqState st = p.seq_state[b];
-    __shared__ double warp_sums[kSampleThreads / 32];
+    __shared__ double warp_sums[kPickScratch];
     __shared__ double s_sums[kWalkChunks];
     __shared__ int s_pick[3];
     __shared__ double s_base[2];
@@ -564,23 +617,7 @@ __global__ void __launch_bounds__(kSampleThreads) shard_pick_kernel(ShardParams 
         for (int i = t; i < n_all; i += kSampleThreads)
             s_sums[i] = sums[(size_t)(i / p.n_chunks) * p.mass_rank_stride + (size_t)b * p.n_chunks + i % p.n_chunks];
         __syncthreads();
-        if (t == 0) {
-            double tot = 0.0;
-            for (int i = 0; i < n_all; ++i) tot += s_sums[i];
-            const double target = (double)p.u_sample[(size_t)b * R + st.n] * tot;
-            int pick = -1, last_pos = -1;
-            double cum = 0.0, base = 0.0;
-            for (int i = 0; i < n_all; ++i) {
-                const double s = s_sums[i];
-                if (s > 0.0) last_pos = i;
-                if (pick < 0 && s > 0.0 && cum + s > target) { pick = i; base = cum; }
-                cum += s;
-            }
-            s_pick[0] = tot > 0.0 ? (pick >= 0 ? pick : last_pos) : -1;
-            s_pick[1] = (pick < 0);
-            s_base[0] = base;
-            s_base[1] = target;
-        }
+        if (t < 32) walk_chunk_masses(s_sums, n_all, (double)p.u_sample[(size_t)b * R + st.n], s_pick, s_base);
         __syncthreads();
         if (s_pick[0] >= 0 || !use_q) break;
         use_q = 0;                             // the residual has no mass (p == q on this row): draw from p
