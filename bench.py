@@ -48,11 +48,11 @@ MIN_SPLIT_STEPS = 5
 # device) and scaled by the K/V bytes of the launch: the kernel streams every K/V byte once, so its
 # traffic grows in proportion.  None: no capture of the kernel as it stands.
 NCU_TRAFFIC_RATIO = {
-    ("attn", "qwen"): 693.4 / 691.5,          # profiles/attn_umma_kernel_qwen7b_long_b16.md (batch 16, scaled by K/V bytes)
+    ("attn", "qwen"): (693.56 + 5.1) / 691.5,  # profiles/attn_umma_kernel_qwen7b_long_b16.md (batch 16, scaled by K/V bytes)
     ("attn", "gemma"): 1.384 / 1.34,          # profiles/attn_split_kernel_gemma12b_b32_t1.md (read 1.378 GB + 6.2 MB written)
     ("lm_head", "qwen"): 1.0934 / 1.0900,     # profiles/lm_head_umma_kernel_qwen7b_b1_t0.md (the weight-bound launches, M <= 256)
     ("lm_head", "gemma"): None,
-    ("residual", "qwen"): (74.39 + 1.85) / 77.86,   # profiles/residual_sample_kernel_qwen7b_lmhead_g5_t1.md
+    ("residual", "qwen"): (74.36 + 2.1) / 77.86,    # profiles/residual_sample_kernel_qwen7b_lmhead_g5_t1.md
     ("residual", "gemma"): None,
 }
 
@@ -267,7 +267,7 @@ def roofline_block(kernel, bound, algorithmic, ms, peaks, peak_src, family):
          "ms_per_launch_best": ms["best"]}
     if bound == "tensor" and peaks.get("bf16_tflops_sustained"):
         r["frac_of_sustained"] = achieved / peaks["bf16_tflops_sustained"]
-    key = {"attn_umma_kernel": "attn", "attn_split_kernel": "attn", "lm_head_umma_kernel": "lm_head",
+    key = {"attn_umma_kernel": "attn", "attn_split_kernel": "attn", "lm_head_umma_kernel": "lm_head", "lm_head_duo_kernel": "lm_head",
            "residual_sample_kernel": "residual"}[kernel]
     ratio = NCU_TRAFFIC_RATIO.get((key, family))
     r["traffic"] = None if (ratio is None or bound == "tensor") else ratio * algorithmic
@@ -378,7 +378,8 @@ def measure(mv, cfg, dev, K, W, attn_kernel, peaks, peak_src, world, sampler=Non
     ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
     attn_name = "attn_umma_kernel" if (attn_kernel == 2 or (attn_kernel == 0 and cfg.head_dim <= 128)) else "attn_split_kernel"
     rl = {"attn": roofline_block(attn_name, "hbm", attn_bytes, t_attn_k, peaks, peak_src, family),
-          "lm_head": roofline_block("lm_head_umma_kernel", "tensor" if cfg.m > ridge else "hbm",
+          # 257 .. 384 token rows take the one-pass kernel (two sub-tiles of the rows in tensor memory at once)
+          "lm_head": roofline_block("lm_head_duo_kernel" if 256 < cfg.m <= 384 else "lm_head_umma_kernel", "tensor" if cfg.m > ridge else "hbm",
                                     lm_flops if cfg.m > ridge else lm_bytes, t_lm, peaks, peak_src, family)}
     rl["attn"]["frac_whole_call"] = attn_bytes / (t_attn["mean"] * 1e-3) / 1e9 / peaks["hbm_gbs"]
     rl["lm_head"]["frac_whole_accept_call"] = rl["lm_head"]["algorithmic"] / (t_accept["mean"] * 1e-3) / \
