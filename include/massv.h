@@ -53,7 +53,9 @@ typedef enum massv_status {
     MASSV_ERR_CAPACITY = -3,      /* page table cannot hold L_b + gamma + 1 positions */
     MASSV_ERR_WORKSPACE = -4,     /* workspace NULL, misaligned or too small */
     MASSV_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed */
-    MASSV_ERR_TIMEOUT = -6        /* device-side wait exceeded its iteration limit (dev_status only) */
+    MASSV_ERR_TIMEOUT = -6,       /* device-side wait exceeded its iteration limit (dev_status only) */
+    MASSV_ERR_BOUNDS = -7         /* debug builds (-DMASSV_DEBUG) only: an index computed on the device fell outside
+                                     its buffer; the access was skipped (dev_status only) */
 } massv_status;
 
 /* Geometry of the attention call. */

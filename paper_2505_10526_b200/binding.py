@@ -14,7 +14,9 @@ import os
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libmassv.so")
+# MASSV_DEBUG=1 selects the build with device-side index checks (same entry points, MASSV_ERR_BOUNDS in dev_status
+# where an index leaves its buffer); it has to exist, like the ordinary library
+LIB_PATH = os.path.join(_PKG, "libmassv_debug.so" if os.environ.get("MASSV_DEBUG", "0") not in ("", "0") else "libmassv.so")
 
 
 class MassvError(RuntimeError):

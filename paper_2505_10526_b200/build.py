@@ -13,6 +13,7 @@ SOURCES = ["api.cu", "attn.cu", "attn_umma.cu", "lm_head.cu", "accept.cu", "acce
 
 
 TEST_LIB = os.path.join(PKG, "libmassv_testhooks.so")
+DEBUG_LIB = os.path.join(PKG, "libmassv_debug.so")
 
 
 def _stale(lib=LIB) -> bool:
@@ -23,15 +24,31 @@ def _stale(lib=LIB) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def _compile(out, extra, verbose=False):
+def _command(out, extra, verbose=False):
     nvcc = os.environ.get("NVCC", "nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC] + extra + \
-          ["-o", out] + [os.path.join(CSRC, s) for s in SOURCES]
+          ["-o", out] + [os.path.join(CSRC, s) for s in SOURCES] + ["-ldl"]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
-    subprocess.run(cmd, check=True)
+    return cmd
+
+
+def _compile(out, extra, verbose=False):
+    subprocess.run(_command(out, extra, verbose), check=True)
     return out
+
+
+VARIANTS = {LIB: [], TEST_LIB: ["-DMASSV_TEST_HOOKS", "-DMASSV_SPIN_LIMIT=65536u"], DEBUG_LIB: ["-DMASSV_DEBUG"]}
+
+
+def build_all(force: bool = False):
+    """The library and its two test variants, the stale ones compiled side by side."""
+    procs = [(lib, subprocess.Popen(_command(lib, extra))) for lib, extra in VARIANTS.items() if force or _stale(lib)]
+    for lib, proc in procs:
+        if proc.wait() != 0:
+            raise subprocess.CalledProcessError(proc.returncode, "nvcc -o " + lib)
+    return list(VARIANTS)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -46,6 +63,14 @@ def build_test_hooks(force: bool = False) -> str:
     if not (force or _stale(TEST_LIB)):
         return TEST_LIB
     return _compile(TEST_LIB, ["-DMASSV_TEST_HOOKS", "-DMASSV_SPIN_LIMIT=65536u"])
+
+
+def build_debug(force: bool = False) -> str:
+    """The same sources with -DMASSV_DEBUG: index checks on the device that record MASSV_ERR_BOUNDS in the status
+    word and skip the access.  The binding loads it instead of the ordinary library when MASSV_DEBUG=1 is set."""
+    if not (force or _stale(DEBUG_LIB)):
+        return DEBUG_LIB
+    return _compile(DEBUG_LIB, VARIANTS[DEBUG_LIB])
 
 
 if __name__ == "__main__":

@@ -390,7 +390,10 @@ __device__ void draw_from_chunk_masses(const AcceptParams& p, int b, const SeqSt
         chunk_masses_global(z_row + (size_t)pick * kResidualChunk, use_q ? q_row + (size_t)pick * kResidualChunk : nullptr,
                             min(kResidualChunk, p.V - pick * kResidualChunk), rc, rr);
         pick_in_chunk(rr, pick * kResidualChunk, s_base[0], s_base[1], warp_sums, s_first, s_last);
-        if (t == 0) *tok_out = (!take_last && *s_first != 0x7fffffff) ? *s_first : *s_last;
+        if (t == 0 && MASSV_IN_BOUNDS(st.n, R, p.dev_status)) {
+            const int tok = (!take_last && *s_first != 0x7fffffff) ? *s_first : *s_last;
+            if (MASSV_IN_BOUNDS(tok, p.V, p.dev_status)) *tok_out = tok;
+        }
     }
     bar_sync_consumers();          // the shared pick state may be reused for this CTA's next sequence
 }
@@ -461,7 +464,7 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
                     double total = 0.0;
 #pragma unroll
                     for (int w = 0; w < kSampleThreads / 32; ++w) total += s_part[s][w];
-                    p.chunk_sums[(size_t)b * p.n_chunks + c] = total;
+                    if (MASSV_IN_BOUNDS((size_t)b * p.n_chunks + c, (size_t)p.B * p.n_chunks, p.dev_status)) p.chunk_sums[(size_t)b * p.n_chunks + c] = total;
                     ++run_cnt;
                     if (kd + 1 == n_items || (item + 1) / p.n_chunks != b) {      // this CTA's last chunk of sequence b
                         __threadfence();

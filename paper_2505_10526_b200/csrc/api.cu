@@ -4,6 +4,8 @@
 
 #include <atomic>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "kernels.cuh"
 
 using namespace massv;
@@ -18,6 +20,13 @@ TimingHooks& timing_hooks() {
 }
 
 namespace {
+
+// A named range around the host side of a call, for timelines (NVTX is header-only: without a tool attached the
+// push and the pop are two null-pointer checks).
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+};
 
 constexpr size_t kAlign = 256;
 
@@ -133,6 +142,7 @@ int massv_verify_attn(const massv_attn_desc* desc, const void* q, const void* k_
                       void* k_pages, void* v_pages, const int32_t* page_table, const int32_t* seq_lens,
                       void* out, float* out_f32, float* lse, void* workspace, size_t workspace_bytes,
                       int32_t* dev_status, massv_stream_t stream) {
+    NvtxRange range("massv_verify_attn");
     const int rc = check_attn_desc(desc);
     if (rc != MASSV_OK) return rc;
     if (!q || !k_new || !v_new || !k_pages || !v_pages || !page_table || !seq_lens || !out) return MASSV_ERR_INVALID_ARG;
@@ -176,6 +186,7 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
                  const float* draft_probs, const float* u_accept, const float* u_sample, int32_t* out_tokens,
                  int32_t* accept_len, float* logits_out, float* probs_out, void* workspace, size_t workspace_bytes,
                  int32_t* dev_status, massv_stream_t stream) {
+    NvtxRange range("massv_accept");
     const int rc = check_accept_desc(desc);
     if (rc != MASSV_OK) return rc;
     const bool sampling = desc->temperature > 0.f;
@@ -470,6 +481,7 @@ int massv_sample_top_p(int32_t rows, int32_t vocab, float temperature, float top
 
 int massv_kv_commit(int32_t batch, int32_t gamma, const int32_t* accept_len, int32_t* seq_lens, int32_t* dev_status,
                     massv_stream_t stream) {
+    NvtxRange range("massv_kv_commit");
     if (batch < 1 || gamma < 0 || !seq_lens) return MASSV_ERR_INVALID_ARG;
     if (gamma > kMaxRows - 1) return MASSV_ERR_UNSUPPORTED;
     return launch_kv_commit(batch, gamma, accept_len, seq_lens, dev_status, reinterpret_cast<cudaStream_t>(stream)) ==
@@ -487,6 +499,7 @@ const char* massv_strerror(int status) {
         case MASSV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case MASSV_ERR_CUDA: return "CUDA call failed";
         case MASSV_ERR_TIMEOUT: return "device-side wait timed out";
+        case MASSV_ERR_BOUNDS: return "device-side index out of bounds (debug build)";
         default: return "unknown status";
     }
 }

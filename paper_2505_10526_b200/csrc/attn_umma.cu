@@ -256,7 +256,8 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             } else {
                 // slot 0: the piece that opens this CTA's range; slot 1: a later piece (it can only be
                 // one that runs on into the next CTA)
-                const size_t slot = (size_t)blockIdx.x * 2 + (f == f_first ? 0 : 1);
+                size_t slot = (size_t)blockIdx.x * 2 + (f == f_first ? 0 : 1);
+                if (!MASSV_IN_BOUNDS(slot, 2 * kFlatMaxCtas, p.dev_status)) slot = 0;
                 sg.part_o = p.flat_part_o + slot * rows_pad * D;
                 sg.part_ml = p.flat_part_ml + slot * rows_pad * 2;
             }
@@ -665,10 +666,13 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             const size_t out1 = r1 < rows ? (((size_t)b * p.R + r1 / G) * p.Hq + g * G + r1 % G) : 0;
             // (Each case has its own loop: this code runs once or twice per CTA, from a cold instruction cache,
             // so what is not executed should not be fetched either.)
+            // (debug build: one decision per warp, because the tensor-memory loads below are warp-wide)
+            const bool rows_in_out = __all_sync(0xffffffffu, MASSV_IN_BOUNDS(out0, (size_t)p.B * p.R * p.Hq, p.dev_status) &&
+                                                                  MASSV_IN_BOUNDS(out1, (size_t)p.B * p.R * p.Hq, p.dev_status));
             if (single) {
                 const float inv0 = 1.f / l_run[0], inv1 = 1.f / l_run[1];
 #pragma unroll 1
-                for (int c0 = 0; c0 < D; c0 += 64) {
+                for (int c0 = 0; c0 < D && rows_in_out; c0 += 64) {
                     uint32_t o[32];
                     tmem_ld_16x64(tmem_o + lane_base + (uint32_t)c0, o);
 #pragma unroll
@@ -721,7 +725,7 @@ attn_umma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constan
             if (lane == 0) mbar_arrive(&o_free_bar);
             if ((lane & 3) == 0) {
                 if (single) {
-                    if (p.lse) {
+                    if (p.lse && rows_in_out) {
                         if (r0 < rows) p.lse[out0] = (m_ref[0] + log2f(l_run[0])) * 0.6931471805599453f;
                         if (r1 < rows) p.lse[out1] = (m_ref[1] + log2f(l_run[1])) * 0.6931471805599453f;
                     }

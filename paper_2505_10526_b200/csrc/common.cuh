@@ -19,6 +19,20 @@ __device__ __forceinline__ void set_status(int32_t* dev_status, int code) {
     if (dev_status) atomicCAS(dev_status, 0, code);
 }
 
+// Index checks of the debug build (-DMASSV_DEBUG): an index outside [0, limit) records MASSV_ERR_BOUNDS in the
+// status word and the guarded access is skipped - no trap, no assert, the context stays usable.  In the ordinary
+// build the macro is the constant true and the checks cost nothing.
+#ifdef MASSV_DEBUG
+__device__ __forceinline__ bool in_bounds_or_report(long long idx, long long limit, int32_t* dev_status) {
+    if (idx >= 0 && idx < limit) return true;
+    set_status(dev_status, MASSV_ERR_BOUNDS);
+    return false;
+}
+#define MASSV_IN_BOUNDS(idx, limit, dev_status) (::massv::in_bounds_or_report((long long)(idx), (long long)(limit), (dev_status)))
+#else
+#define MASSV_IN_BOUNDS(idx, limit, dev_status) (true)
+#endif
+
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t h) {
     return __uint_as_float(((uint32_t)h) << 16);
 }

@@ -49,6 +49,7 @@ struct UmmaParams {
     float* logits;       // [M, V] or nullptr
     float *part_max, *part_sum;
     int32_t* part_idx;
+    int n_part = 0;      // partial slots behind part_max / part_sum / part_idx (the debug build checks the slot index)
     int32_t* dev_status;
     int idx_offset;      // added to the argmax indices that leave the kernel
     int test_skip_stage = 0;   // test builds only: withhold the second K block of the first tile
@@ -487,9 +488,11 @@ lm_head_umma_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_c
             for (int qd = 1; qd < 4; ++qd)
                 acc = stat_combine(acc, Stat{run_m[qd][c], run_s[qd][c], run_i[qd][c]}, p.scale_log2, p.greedy != 0);
             const size_t slot = (size_t)(PAIR ? group * 2 + (int)pair_rank : group) * p.M;
-            p.part_max[slot + tok] = acc.m;
-            p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
-            p.part_idx[slot + tok] = acc.idx == 0x7fffffff ? acc.idx : acc.idx + p.idx_offset;
+            if (MASSV_IN_BOUNDS(slot + tok, (size_t)p.n_part * p.M, p.dev_status)) {
+                p.part_max[slot + tok] = acc.m;
+                p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
+                p.part_idx[slot + tok] = acc.idx == 0x7fffffff ? acc.idx : acc.idx + p.idx_offset;
+            }
         }
     }
     if constexpr (PAIR) cluster_sync_all();      // neither CTA frees TMEM or leaves while the other may still use it
@@ -848,9 +851,11 @@ lm_head_duo_kernel(const __grid_constant__ CUtensorMap map_w128, const __grid_co
             for (int qd = 1; qd < 4; ++qd)
                 acc = stat_combine(acc, Stat{run_m[qd][c], run_s[qd][c], run_i[qd][c]}, p.scale_log2, p.greedy != 0);
             const size_t slot = (size_t)(group * 2 + (int)pair_rank) * p.M;
-            p.part_max[slot + tok] = acc.m;
-            p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
-            p.part_idx[slot + tok] = acc.idx == 0x7fffffff ? acc.idx : acc.idx + p.idx_offset;
+            if (MASSV_IN_BOUNDS(slot + tok, (size_t)p.n_part * p.M, p.dev_status)) {
+                p.part_max[slot + tok] = acc.m;
+                p.part_sum[slot + tok] = p.greedy ? 0.f : acc.s;
+                p.part_idx[slot + tok] = acc.idx == 0x7fffffff ? acc.idx : acc.idx + p.idx_offset;
+            }
         }
     }
     cluster_sync_all();      // neither CTA frees TMEM or leaves while the other may still use it
@@ -931,7 +936,7 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.greedy = q.greedy;
     p.scale_log2 = q.inv_T_log2e;
     p.logits = q.logits;
-    p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
+    p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx; p.n_part = q.n_part;
     p.dev_status = q.dev_status;
     p.idx_offset = q.idx_offset;
     p.test_skip_stage = q.test_skip_stage;
@@ -963,7 +968,7 @@ cudaError_t launch_lm_head(const LmHeadParams& q, cudaStream_t stream, int* n_pa
     p.greedy = q.greedy;
     p.scale_log2 = q.inv_T_log2e;
     p.logits = q.logits;
-    p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx;
+    p.part_max = q.part_max; p.part_sum = q.part_sum; p.part_idx = q.part_idx; p.n_part = q.n_part;
     p.dev_status = q.dev_status;
     p.idx_offset = q.idx_offset;
     const int slots = groups * (pair ? 2 : 1);

@@ -33,6 +33,16 @@ def test_every_declared_symbol_is_exported(mv):
         assert hasattr(lib, n), n
 
 
+def test_the_test_and_debug_builds_export_the_same_symbols(mv):
+    pkg_dir = os.path.dirname(mv.LIB_PATH)
+    for variant in ("libmassv_testhooks.so", "libmassv_debug.so"):
+        lib = ctypes.CDLL(os.path.join(pkg_dir, variant))
+        for n in declared_symbols():
+            assert hasattr(lib, n), (variant, n)
+        lib.massv_strerror.restype = ctypes.c_char_p
+        assert b"bounds" in lib.massv_strerror(-7)
+
+
 def test_python_binding_has_the_same_names(mv):
     for n in declared_symbols():
         assert hasattr(mv, n) or hasattr(mv.binding, n), n
