@@ -46,3 +46,27 @@ def test_config_table_covers_the_five_benchmark_shapes():
         assert n in CONFIGS
     c = get_config("gemma12b_b32_t1")
     assert (c.n_q_heads, c.n_kv_heads, c.head_dim, c.hidden, c.vocab) == (16, 8, 256, 3840, 262144)
+
+
+def test_philox_matches_the_published_known_answers():
+    """Philox4x32-10 known-answer vectors (Salmon et al., SC 2011, the reference test vectors of the algorithm):
+    counter and key all zero, all ones, and the digits of pi."""
+    from workloads.philox import philox4x32_10, uniforms
+    cases = [([0, 0, 0, 0], (0, 0), [0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8]),
+             ([0xffffffff] * 4, (0xffffffff, 0xffffffff), [0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd]),
+             ([0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344], (0xa4093822, 0x299f31d0),
+              [0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1])]
+    for counter, key, want in cases:
+        got = philox4x32_10(np.array([counter], dtype=np.uint32), key)[0]
+        assert got.tolist() == want
+    u = uniforms(100003, 7, 1)
+    assert u.dtype == np.float32 and u.min() >= 0.0 and u.max() < 1.0 and abs(float(u.mean()) - 0.5) < 5e-3
+    assert np.array_equal(u[:10], uniforms(10, 7, 1)) and not np.array_equal(u[:10], uniforms(10, 7, 0)[:10])
+
+
+def test_uniforms_do_not_depend_on_the_device_the_workload_is_built_on():
+    from workloads.philox import uniforms
+    cfg = get_config("tiny_t1")
+    w = generate(cfg)
+    assert np.array_equal(w["u_accept"].numpy().ravel(), uniforms(cfg.batch * cfg.gamma, cfg.seed, 0))
+    assert np.array_equal(w["u_sample"].numpy().ravel(), uniforms(cfg.batch * cfg.rows, cfg.seed, 1))

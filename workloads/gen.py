@@ -2,7 +2,9 @@
 
 Every tensor is drawn from one ``torch.Generator`` seeded with the config's
 seed, in a fixed order, on the requested device (the CPU generator and the CUDA
-Philox generator give different streams; each is reproducible on its own).
+generator give different streams; each is reproducible on its own), except the
+uniforms of the acceptance tests and of the draw: those come from Philox4x32-10
+keyed by the seed (workloads/philox.py) and are the same on either device.
 Values destined for bf16 tensors are drawn in fp32 and rounded once
 (round-to-nearest-even), so every consumer sees the same bf16 bits.
 
@@ -16,6 +18,7 @@ import math
 
 import torch
 
+from . import philox
 from .configs import VerifyConfig
 
 PAGE_SIZE = 16
@@ -118,6 +121,8 @@ def generate(cfg: VerifyConfig, device="cpu", with_lm_head=True, with_attention=
         else:
             tok = zq.argmax(dim=-1)
         out["draft_tokens"] = tok.to(torch.int32).contiguous()
-        out["u_accept"] = torch.rand((B, g), generator=gen, device=dev, dtype=torch.float32)
-        out["u_sample"] = torch.rand((B, R), generator=gen, device=dev, dtype=torch.float32)
+        # the uniforms of the rejection tests and of the draw: Philox4x32-10 keyed by the config's seed, so the
+        # same numbers on either device (stream 0: acceptance, stream 1: draw)
+        out["u_accept"] = torch.from_numpy(philox.uniforms(B * g, cfg.seed, 0)).view(B, g).to(dev)
+        out["u_sample"] = torch.from_numpy(philox.uniforms(B * R, cfg.seed, 1)).view(B, R).to(dev)
     return out
