@@ -26,6 +26,7 @@ constexpr int kResidualCtasPerSm = 2;
 constexpr int kResidualSeqCache = 8; // sequences whose scan results a CTA keeps in shared memory
 constexpr int kWalkChunks = 512;  // chunk masses staged in shared memory for the walk (vocabularies up to 2M entries)
 static_assert(kPerThread == 16, "chunk layout");
+static_assert(kSampleThreads / 32 == kResidualSegments, "one consumer warp per segment of a chunk");
 
 struct Stat {
     float m;   // running max logit
@@ -398,6 +399,120 @@ __device__ void draw_from_chunk_masses(const AcceptParams& p, int b, const SeqSt
     bar_sync_consumers();          // the shared pick state may be reused for this CTA's next sequence
 }
 
+// The same draw by ONE warp, for callers that kept the masses of every chunk's eight 512-entry segments
+// (seg_sums): chunk masses -> chunk, its eight segment masses -> segment, the segment's 512 entries (16 contiguous
+// ones per lane) -> token.  Three dependent reads of a few KB instead of a 32 KB chunk and four barriers of 256
+// threads, and little code: this runs once per sequence at the very end of the kernel, when nothing hides its
+// latency.  Returns false (in every lane) where the residual has no mass at all: the caller then takes the
+// path above, which knows the fall-back to p.
+__device__ __forceinline__ bool draw_by_one_warp(const AcceptParams& p, int b, const SeqState& st, float inv_T) {
+    const int lane = threadIdx.x & 31, R = p.gamma + 1;
+    const double* sums = p.chunk_sums + (size_t)b * p.n_chunks;
+    // 1. the chunk: lane l owns a contiguous run of chunks
+    const int per = (p.n_chunks + 31) / 32;
+    const int i0 = min(p.n_chunks, lane * per), i1 = min(p.n_chunks, i0 + per);
+    double local = 0.0;
+    for (int i = i0; i < i1; ++i) local += __ldcg(sums + i);
+    double incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double y = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += y;
+    }
+    const double tot = __shfl_sync(0xffffffffu, incl, 31);
+    if (!(tot > 0.0)) return false;
+    const double target = (double)p.u_sample[(size_t)b * R + st.n] * tot;
+    double run = incl - local, my_base = 0.0;
+    int my_pick = 0x7fffffff, my_last = -1;
+    for (int i = i0; i < i1; ++i) {
+        const double sm = __ldcg(sums + i);
+        if (sm > 0.0) {
+            my_last = i;
+            if (my_pick == 0x7fffffff && run + sm > target) { my_pick = i; my_base = run; }
+        }
+        run += sm;
+    }
+    const unsigned found = __ballot_sync(0xffffffffu, my_pick != 0x7fffffff);
+    const int last_pos = __reduce_max_sync(0xffffffffu, my_last);
+    const int src = found ? __ffs(found) - 1 : 0;
+    const int chunk = found ? __shfl_sync(0xffffffffu, my_pick, src) : last_pos;
+    double base = found ? __shfl_sync(0xffffffffu, my_base, src) : 0.0;
+    bool take_last = !found;            // rounding pushed the target past the end: the last positive entry
+    // 2. the segment inside the chunk: every lane walks the same eight masses
+    const double* seg = p.seg_sums + ((size_t)b * p.n_chunks + chunk) * kResidualSegments;
+    double sg[kResidualSegments];
+#pragma unroll
+    for (int j = 0; j < kResidualSegments; ++j) sg[j] = __ldcg(seg + j);
+    int seg_pick = -1, seg_last = -1;
+    double seg_base = base;
+    {
+        double r = base;
+#pragma unroll
+        for (int j = 0; j < kResidualSegments; ++j) {
+            if (sg[j] > 0.0) {
+                seg_last = j;
+                if (!take_last && seg_pick < 0 && r + sg[j] > target) { seg_pick = j; seg_base = r; }
+            }
+            r += sg[j];
+        }
+    }
+    if (seg_pick < 0) { seg_pick = seg_last; take_last = true; }
+    // 3. the token inside the segment: 16 contiguous entries per lane
+    const RowCtx rc(st, inv_T);
+    const int e0 = chunk * kResidualChunk + seg_pick * (kResidualChunk / kResidualSegments) + lane * 16;
+    const float* z = p.logits + (size_t)(b * R + st.n) * p.V + e0;
+    const float* q = st.use_q ? p.draft_probs + ((size_t)b * p.gamma + st.n) * p.V + e0 : nullptr;
+    float m[16];
+    float4 zz[4], qq[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        zz[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        qq[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e0 + 4 * k < p.V) {                      // V is a multiple of 4: a group exists whole or not at all
+            zz[k] = __ldcg(reinterpret_cast<const float4*>(z) + k);
+            if (q) qq[k] = __ldg(reinterpret_cast<const float4*>(q) + k);
+        }
+    }
+    double lane_sum = 0.0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const float zs[4] = {zz[k].x, zz[k].y, zz[k].z, zz[k].w}, qs[4] = {qq[k].x, qq[k].y, qq[k].z, qq[k].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float v = 0.f;
+            if (e0 + 4 * k < p.V) {
+                const float pv = rc.prob(zs[e]);
+                v = q ? fmaxf(pv - qs[e], 0.f) : pv;
+            }
+            m[4 * k + e] = v;
+            lane_sum += (double)v;
+        }
+    }
+    double lincl = lane_sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double y = __shfl_up_sync(0xffffffffu, lincl, o);
+        if (lane >= o) lincl += y;
+    }
+    double r = seg_base + (lincl - lane_sum);
+    int first = 0x7fffffff, last = -1;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        r += (double)m[i];
+        if (m[i] > 0.f) {
+            last = e0 + i;
+            if (first == 0x7fffffff && r > target) first = e0 + i;
+        }
+    }
+    const int tok_first = __reduce_min_sync(0xffffffffu, first);
+    const int tok_last = __reduce_max_sync(0xffffffffu, last);
+    if (lane == 0 && MASSV_IN_BOUNDS(st.n, R, p.dev_status)) {
+        const int tok = (!take_last && tok_first != 0x7fffffff) ? tok_first : tok_last;
+        if (tok >= 0 && MASSV_IN_BOUNDS(tok, p.V, p.dev_status)) p.out_tokens[(size_t)b * R + st.n] = tok;
+    }
+    return true;
+}
+
 // T > 0: the extra token of every sequence, one pass over the single row it is drawn from.  Work item =
 // (sequence, 4096-entry chunk); a persistent grid of one wave deals the items out in contiguous runs.
 // Warp 8 is the producer: it keeps a ring of items filled with bulk copies (the chunk of the row's logits
@@ -464,7 +579,14 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
                     double total = 0.0;
 #pragma unroll
                     for (int w = 0; w < kSampleThreads / 32; ++w) total += s_part[s][w];
-                    if (MASSV_IN_BOUNDS((size_t)b * p.n_chunks + c, (size_t)p.B * p.n_chunks, p.dev_status)) p.chunk_sums[(size_t)b * p.n_chunks + c] = total;
+                    if (MASSV_IN_BOUNDS((size_t)b * p.n_chunks + c, (size_t)p.B * p.n_chunks, p.dev_status)) {
+                        p.chunk_sums[(size_t)b * p.n_chunks + c] = total;
+                        if (p.seg_sums) {       // the eight warps' shares are the chunk's eight segments, in vocabulary order
+                            double2* sg = reinterpret_cast<double2*>(p.seg_sums + ((size_t)b * p.n_chunks + c) * kResidualSegments);
+#pragma unroll
+                            for (int w = 0; w < kSampleThreads / 32; w += 2) sg[w / 2] = make_double2(s_part[s][w], s_part[s][w + 1]);
+                        }
+                    }
                     ++run_cnt;
                     if (kd + 1 == n_items || (item + 1) / p.n_chunks != b) {      // this CTA's last chunk of sequence b
                         __threadfence();
@@ -542,6 +664,17 @@ __global__ void __launch_bounds__(kResidualThreads, kResidualCtasPerSm) residual
     const int n_pending = s_n_pending;
     for (int i = 0; i < n_pending; ++i) {
         const int b = s_pending[i];
+        if (p.seg_sums) {
+            // one warp makes the draw from the segment masses; the others join only if the residual turns out empty
+            if (warp == 0) {
+                const bool done = draw_by_one_warp(p, b, state_of(b), inv_T);
+                if (lane == 0) s_pick[0] = done ? 1 : 0;
+            }
+            bar_sync_consumers();
+            const bool done = s_pick[0] != 0;
+            bar_sync_consumers();
+            if (done) continue;
+        }
         draw_from_chunk_masses(p, b, state_of(b), inv_T, warp_sums, s_sums, s_pick, s_base, &s_first, &s_last);
     }
 }

@@ -107,7 +107,7 @@ int check_accept_desc(const massv_accept_desc* d) {
 
 struct AcceptLayout {
     int n_part, n_chunks;
-    size_t off_max, off_sum, off_idx, off_state, off_chunks, off_counters, off_rowstat, off_logits, total;
+    size_t off_max, off_sum, off_idx, off_state, off_chunks, off_segs, off_counters, off_rowstat, off_logits, total;
 };
 
 AcceptLayout accept_layout(const massv_accept_desc& d) {
@@ -121,6 +121,8 @@ AcceptLayout accept_layout(const massv_accept_desc& d) {
     l.off_idx = off; off += align_up((size_t)l.n_part * M * sizeof(int32_t), kAlign);
     l.off_state = off; off += align_up((size_t)d.batch * sizeof(SeqState), kAlign);
     l.off_chunks = off; off += align_up((size_t)d.batch * l.n_chunks * sizeof(double), kAlign);
+    l.off_segs = off;
+    if (d.temperature > 0.f) off += align_up((size_t)d.batch * l.n_chunks * kResidualSegments * sizeof(double), kAlign);
     l.off_counters = off; off += align_up((size_t)d.batch * sizeof(unsigned int), kAlign);
     l.off_rowstat = off; off += align_up(M * 2 * sizeof(float), kAlign);
     l.off_logits = off;
@@ -230,6 +232,7 @@ int massv_accept(const massv_accept_desc* desc, const void* hidden, const void* 
     a.out_tokens = out_tokens; a.accept_len = accept_len; a.probs_out = probs_out;
     a.seq_state = reinterpret_cast<SeqState*>(ws + l.off_state);
     a.chunk_sums = reinterpret_cast<double*>(ws + l.off_chunks);
+    a.seg_sums = desc->temperature > 0.f ? reinterpret_cast<double*>(ws + l.off_segs) : nullptr;
     a.counters = reinterpret_cast<unsigned int*>(ws + l.off_counters);
     a.row_stats = reinterpret_cast<float*>(ws + l.off_rowstat);
     a.n_chunks = l.n_chunks;

@@ -13,6 +13,7 @@ constexpr int kPageSize = 16;       // tokens per KV page
 constexpr int kMaxRows = 8;         // gamma + 1 <= 8
 constexpr int kVocabTile = 128;     // vocabulary rows per LM-head tile
 constexpr int kResidualChunk = 4096;  // vocabulary entries per residual-mass chunk
+constexpr int kResidualSegments = 8;  // a chunk is eight segments of 512 entries, one per consumer warp of the draw kernel
 
 // Record the first device-side problem without trapping.
 __device__ __forceinline__ void set_status(int32_t* dev_status, int code) {

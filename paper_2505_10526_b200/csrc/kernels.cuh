@@ -77,6 +77,7 @@ struct AcceptParams {
     SeqState* seq_state;            // [B]
     float* row_stats = nullptr;     // optional [B*(gamma+1), 2]: the merged (max logit, sum exp((z - max)/T)) of every row
     double* chunk_sums;             // [B, n_chunks]
+    double* seg_sums = nullptr;     // optional [B, n_chunks, 8]: the masses of the eight 512-entry segments of every chunk
     unsigned int* counters;         // [B]
     int n_chunks;
     int32_t* dev_status;
