@@ -52,7 +52,7 @@ NCU_TRAFFIC_RATIO = {
     ("attn", "gemma"): 1.384 / 1.34,          # profiles/attn_split_kernel_gemma12b_b32_t1.md (read 1.378 GB + 6.2 MB written)
     ("lm_head", "qwen"): 1.0934 / 1.0900,     # profiles/lm_head_umma_kernel_qwen7b_b1_t0.md (the weight-bound launches, M <= 256)
     ("lm_head", "gemma"): (2.04587 + 0.14472) / 2.01474,   # profiles/lm_head_umma_kernel_gemma12b_b32_t1.md (weights once + the fp32 logits that left L2)
-    ("residual", "qwen"): (74.36 + 2.1) / 77.86,    # profiles/residual_sample_kernel_qwen7b_lmhead_g5_t1.md
+    ("residual", "qwen"): (74.30 + 1.35) / 77.86,   # profiles/residual_sample_kernel_qwen7b_lmhead_g5_t1.md
     ("residual", "gemma"): (62.98 + 0.12) / 67.11,    # profiles/lm_head_umma_kernel_gemma12b_b32_t1.md (second table)
 }
 
