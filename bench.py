@@ -51,9 +51,9 @@ NCU_TRAFFIC_RATIO = {
     ("attn", "qwen"): (693.56 + 5.1) / 691.5,  # profiles/attn_umma_kernel_qwen7b_long_b16.md (batch 16, scaled by K/V bytes)
     ("attn", "gemma"): 1.384 / 1.34,          # profiles/attn_split_kernel_gemma12b_b32_t1.md (read 1.378 GB + 6.2 MB written)
     ("lm_head", "qwen"): 1.0934 / 1.0900,     # profiles/lm_head_umma_kernel_qwen7b_b1_t0.md (the weight-bound launches, M <= 256)
-    ("lm_head", "gemma"): (2.04587 + 0.14472) / 2.01474,   # profiles/lm_head_umma_kernel_gemma12b_b32_t1.md (weights once + the fp32 logits that left L2)
+    ("lm_head", "gemma"): (2.04619 + 0.14287) / 2.01474,   # profiles/lm_head_umma_kernel_gemma12b_b32_t1.md (weights once + the fp32 logits that left L2)
     ("residual", "qwen"): (74.30 + 1.35) / 77.86,   # profiles/residual_sample_kernel_qwen7b_lmhead_g5_t1.md
-    ("residual", "gemma"): (62.98 + 0.12) / 67.11,    # profiles/lm_head_umma_kernel_gemma12b_b32_t1.md (second table)
+    ("residual", "gemma"): (62.99 + 0.08) / 67.11,    # profiles/lm_head_umma_kernel_gemma12b_b32_t1.md (second table)
 }
 
 
